@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the budgeted MoE verify layer (MoE-Spec, Algorithm 1) on B200.
+
+A "step" is one pass of the whole hot path (router -> shortlist -> re-routing ->
+gather -> expert FFNs over the kept experts -> combine) over one draft tree.
+Workload at N=1: the OLMoE-shaped single layer (d=2048, N=64, k=8, f=1024,
+bf16 weights, fp32 accumulation), M=63 tree tokens, budget B=32; the other
+budgets of that configuration are reported in "sweep".  Inputs are seeded and
+synthetic.  L2 reuse is defeated by rotating over independently seeded copies
+of the layer (each step streams ~400 MB; 126 MB of L2 cannot hold a copy).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints one JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
+independent replica of the same workload on its own GPU (the layer has no
+data-path collective); time is the max over ranks.  --impl reference times the
+CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2602_16052_b200 import synth
+
+METRIC = "us per budgeted MoE verify layer and achieved HBM GB/s (% roofline) vs M, B"
+WORKLOAD = "olmoe"
+M_TOKENS = 63
+B_HEADLINE = 32
+N_COPIES = 4
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of the two expert-FFN launches of one
+# verify layer (M=63, B=32), from the ncu capture summarised under profiles/; None until captured
+FFN_DRAM_TRAFFIC_BYTES = None
+
+
+def workload_name(cfg):
+    return (f"{WORKLOAD} single layer d={cfg.d} N={cfg.n_experts} k={cfg.k} f={cfg.f} M={M_TOKENS} B={B_HEADLINE} "
+            f"substitution renormalised, bf16 weights, fp32 accumulate and output")
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def mark(self):
+        return time.time()
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if (t0 is None or t >= t0 - 0.05) and (t1 is None or t <= t1 + 0.15)]
+        if not rows:
+            rows = [l for _, l in self.lines]
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            parts = [x.strip() for x in l.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(cfg, M, n_active, out_bytes):
+    """Bytes the method itself must move for one layer: kept experts' weights, the router, hidden in, out."""
+    w = 2 if cfg.dtype == "bf16" else 4
+    return n_active * 3 * cfg.d * cfg.f * w + cfg.n_experts * cfg.d * w + M * cfg.d * w + M * cfg.d * out_bytes
+
+
+def build_layers(cfg, M, n_copies, device, out_dtype):
+    from paper_2602_16052_b200 import moespec
+    layers, hiddens = [], []
+    for c in range(n_copies):
+        L = synth.gen_layer(cfg, seed=1000 + c, layer=0, device=device)
+        hiddens.append(synth.gen_hidden(cfg, M, seed=1000 + c, layer=0, device=device))
+        layers.append(moespec.Layer(L["router_w"], L["router_bias"], L["w_gate"], L["w_up"], L["w_down"], max_M=M,
+                                    max_k=cfg.k, policy=moespec.SUBSTITUTION, shortlist=moespec.FROM_ALL,
+                                    renormalize=True, out_dtype=out_dtype))
+    return layers, hiddens
+
+
+def time_steps(layers, hiddens, outs, k, B, steps, warmup, barrier):
+    """W untimed steps, then exactly K steps between two events on the launching stream."""
+    n = len(layers)
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        layers[i % n].verify_layer(hiddens[i % n], k, B, outs[i % n], stream)
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        layers[i % n].verify_layer(hiddens[i % n], k, B, outs[i % n], stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    return e0.elapsed_time(e1)  # ms
+
+
+def time_e2e(layers, hiddens, k, B, steps, warmup, out_dtype):
+    """Same metric through the host-buffer entry point: H2D of the step's hidden states and D2H of its
+    result are inside the timed region of every step."""
+    n = len(layers)
+    h_host = [h.cpu().pin_memory() for h in hiddens]
+    o_host = [torch.empty(h.shape, dtype=out_dtype).pin_memory() for h in hiddens]
+    for i in range(warmup):
+        layers[i % n].verify_layer_host(h_host[i % n], k, B, o_host[i % n])
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(steps):
+        layers[i % n].verify_layer_host(h_host[i % n], k, B, o_host[i % n])   # synchronises inside
+    t1 = time.perf_counter()
+    h2d = h_host[0].numel() * h_host[0].element_size()
+    d2h = o_host[0].numel() * o_host[0].element_size()
+    return (t1 - t0) * 1e3, h2d, d2h
+
+
+def kernel_profile(layers, hiddens, outs, k, B, reps):
+    """Average per-kernel duration with the library's event bracketing (separate from the timed region)."""
+    n = len(layers)
+    acc = {}
+    for L in layers:
+        L.set_profiling(True)
+    for i in range(reps + 3):
+        L = layers[i % n]
+        L.verify_layer(hiddens[i % n], k, B, outs[i % n])
+        t = L.get_kernel_times()
+        if i >= 3:
+            for name, ms in t.items():
+                acc.setdefault(name, []).append(ms)
+    for L in layers:
+        L.set_profiling(False)
+    return {name: sum(v) / len(v) for name, v in acc.items()}
+
+
+def oracle_case(cfg, M, seed):
+    L = synth.gen_layer(cfg, seed=seed, layer=0, device="cpu")
+    h = synth.gen_hidden(cfg, M, seed=seed, layer=0, device="cpu")
+    f64 = lambda t: t.to(torch.float64).numpy()
+    return {k: f64(v) for k, v in L.items()}, f64(h)
+
+
+def time_oracle(cfg, M, B, min_seconds, max_reps, case=None):
+    """The CPU oracle as it stands on the host cores: whole layers of the same workload until the
+    sample has used about `min_seconds` of wall time (at most max_reps layers)."""
+    from oracle import moespec_oracle as orc
+    L, h = case or oracle_case(cfg, M, seed=1000)
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [os.cpu_count() or 1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    times = []
+    t_start = time.perf_counter()
+    while len(times) < max_reps and (not times or time.perf_counter() - t_start < min_seconds):
+        t0 = time.perf_counter()
+        orc.verify_layer(h, L["router_w"], L["router_bias"], L["w_gate"], L["w_up"], L["w_down"], cfg.k, B,
+                         orc.SUBSTITUTION, orc.FROM_ALL, True)
+        times.append(time.perf_counter() - t0)
+    return statistics.median(times) * 1e6, cores, len(times)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = synth.CONFIGS[WORKLOAD]
+    case = oracle_case(cfg, M_TOKENS, seed=1000)
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(cfg, M_TOKENS, B_HEADLINE, 0.0, 1, case)
+    steps = max(1, min(args.steps, 5))
+    us, cores, reps = time_oracle(cfg, M_TOKENS, B_HEADLINE, 1e9, steps, case)
+    sample = f"{reps} whole verify layers (M={M_TOKENS}, B={B_HEADLINE}) of the same workload, median"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": reps,
+        "warmup": min(args.warmup, 1), "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(cfg)},
+        "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": us, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="moespec", choices=["moespec", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        torch.cuda.set_device(0)
+        local_rank = 0
+    device = torch.device("cuda", local_rank)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    def max_over_ranks(x: float) -> float:
+        if dist is None:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    cfg = synth.CONFIGS[WORKLOAD]
+    M, k, B = M_TOKENS, cfg.k, B_HEADLINE
+    out_dtype = torch.float32          # unrounded fp32 accumulators, the output the 2e-2*RMS bar is stated on
+    layers, hiddens = build_layers(cfg, M, N_COPIES, device, out_dtype)
+    outs = [torch.empty((M, cfg.d), dtype=out_dtype, device=device) for _ in layers]
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    t_mark0 = sampler.mark()
+    ms_total = time_steps(layers, hiddens, outs, k, B, args.steps, args.warmup, barrier)
+    t_mark1 = sampler.mark()
+    clocks = sampler.stop(t_mark0, t_mark1)
+    ms_total = max_over_ranks(ms_total)
+    launches_per_step = layers[0].last_launch_count()
+    stats = layers[0].get_stats()
+    assert stats["status"] == 0, stats
+
+    e2e_ms, h2d, d2h = time_e2e(layers, hiddens, k, B, args.steps, args.warmup, out_dtype)
+    e2e_ms = max_over_ranks(e2e_ms)
+
+    # value: job-wide microseconds per verify layer (all ranks' layers / max time over ranks)
+    us_per_layer = ms_total * 1e3 / (args.steps * world)
+    e2e_us = e2e_ms * 1e3 / (args.steps * world)
+
+    # roofline of the dominant kernel: the expert-FFN weight stream (two launches of ffn_tc_kernel per layer)
+    peak, peak_kind = measured_peaks()
+    kt = kernel_profile(layers, hiddens, outs, k, B, reps=40)
+    n_active = [L.get_stats()["n_active"] for L in layers]
+    mean_active = sum(n_active) / len(n_active)
+    ffn_bytes = mean_active * cfg.expert_weight_bytes()
+    ffn_ms = kt["ffn_gate_up"] + kt["ffn_down"]
+    achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
+    layer_bytes = algorithmic_bytes(cfg, M, mean_active, 4)
+    roofline = {
+        "bound": "hbm", "kernel": "ffn_tc_kernel (gate/up launch + down launch)",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+        "traffic": FFN_DRAM_TRAFFIC_BYTES,
+        "algorithmic_bytes_per_layer": ffn_bytes, "kernel_us": {n: v * 1e3 for n, v in kt.items()},
+        "gate_up_GBs": mean_active * 2 * cfg.d * cfg.f * 2 / (kt["ffn_gate_up"] * 1e-3) / 1e9,
+        "down_GBs": mean_active * cfg.d * cfg.f * 2 / (kt["ffn_down"] * 1e-3) / 1e9,
+        "whole_layer": {"bytes": layer_bytes, "GBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9,
+                        "frac": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / peak,
+                        "frac_of_nominal_8TBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / 8000.0},
+    }
+
+    sweep = []
+    if not args.no_sweep:
+        for Bs in synth.SWEEPS[WORKLOAD]["B"]:
+            ms_b = time_steps(layers, hiddens, outs, k, Bs, max(20, args.steps // 4), 5, barrier)
+            act = sum(L.get_stats()["n_active"] for L in layers) / len(layers)
+            us_b = ms_b * 1e3 / max(20, args.steps // 4)
+            by = algorithmic_bytes(cfg, M, act, 4)
+            sweep.append({"M": M, "B": Bs, "us": us_b, "n_active": act, "GBs": by / (us_b * 1e-6) / 1e9,
+                          "frac": by / (us_b * 1e-6) / 1e9 / peak})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        us, cores, reps = time_oracle(cfg, M, B, 10.0, 6)
+        cpu = {"value": us, "unit": "us", "cores": cores, "kind": "oracle",
+               "sample": f"{reps} whole verify layers (M={M}, B={B}) of the same workload, median"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": us_per_layer, "unit": "us", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg),
+                       "l2": f"rotating over {N_COPIES} independently seeded layer copies "
+                             f"({N_COPIES * cfg.n_experts * cfg.expert_weight_bytes() / 1e9:.1f} GB); each step streams "
+                             f"{ffn_bytes / 1e6:.0f} MB > 126 MB L2",
+                       "replicas": world, "n_active": mean_active, "n_union": stats["n_union"],
+                       "coverage": stats["coverage"]},
+            "clocks": clocks,
+            "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+            "sweep": sweep,
+        }
+        print(json.dumps(line), flush=True)
+    for L in layers:
+        L.destroy()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

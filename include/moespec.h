@@ -1,0 +1,181 @@
+/*
+ * moespec.h - C ABI of the budgeted MoE verify layer (MoE-Spec, Algorithm 1).
+ *
+ * One call runs, for M draft-tree tokens, the whole layer the target model
+ * executes while verifying a speculative draft tree:
+ *   router projection and softmax (Eq. 1) -> per-token top-k (Eq. 2) ->
+ *   per-expert score s_i = sum_t g_i(h_t) (Eq. 5) -> shortlist S of the B best
+ *   experts (Section 3.2) -> per-token re-routing under the substitution (Eq. 8)
+ *   or truncation (Eq. 7) policy with the mixing weights of Section 3.3 ->
+ *   per-expert gather (Appendix C) -> SwiGLU expert FFNs over the kept experts
+ *   only -> gate-weighted combine (outer sums of Eq. 7 / Eq. 8).
+ * Every step runs in CUDA kernels for sm_100a.  There is no CPU path.
+ *
+ * Conventions
+ *   - All functions return 0 on success and a negative moespec_status on error.
+ *     Nothing throws, aborts or traps the device.
+ *   - "device" pointers are CUDA device memory of the layer's device; "host"
+ *     pointers are ordinary host memory.  The library never takes ownership of a
+ *     caller's buffer.  Weight, bias, hidden and out buffers are borrowed; weights
+ *     and bias must stay valid and unchanged for the lifetime of the handle.
+ *   - verify/route calls only enqueue work on the given stream and return; they
+ *     do not synchronise (the *_host variant and the get_* calls do).
+ *   - One call in flight per handle: the handle owns one workspace.
+ *   - Argument rules: 0 <= M <= max_M (M = 0 is a no-op); 1 <= k <= min(N, max_k);
+ *     B >= 1, B > N is clamped to N (B = N is the unbudgeted layer); B < k is legal
+ *     (substitution then gives each token min(k, |S|) experts).
+ *   - Rankings everywhere order by (key descending, expert index ascending).
+ *     Per-token rankings use the fp32 logit as key; the shortlist uses the fp64
+ *     score.  Inputs must be finite.
+ */
+#ifndef MOESPEC_H_
+#define MOESPEC_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moespec_layer moespec_layer_t; /* opaque, created and freed by the library */
+
+typedef enum {
+  MOESPEC_OK = 0,
+  MOESPEC_ERR_INVALID_ARG = -1,   /* a size, enum or flag outside its documented range          */
+  MOESPEC_ERR_NULL_POINTER = -2,  /* a required pointer was NULL                                 */
+  MOESPEC_ERR_UNSUPPORTED = -3,   /* legal request the kernels do not cover (alignment, shapes)  */
+  MOESPEC_ERR_OUT_OF_MEMORY = -4, /* workspace allocation failed                                 */
+  MOESPEC_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed (see moespec_last_cuda_error) */
+  MOESPEC_ERR_TIMEOUT = -6,       /* a bounded device-side wait expired (reported via stats)     */
+  MOESPEC_ERR_INTERNAL = -7,      /* a device-side consistency check failed (reported via stats) */
+  MOESPEC_ERR_BAD_HANDLE = -8     /* handle is NULL, was destroyed, or was never created         */
+} moespec_status;
+
+typedef enum { MOESPEC_BF16 = 1, MOESPEC_FP32 = 2 } moespec_dtype_t;
+/* Token policy of Section 3.3: Eq. 8 / Eq. 7. */
+typedef enum { MOESPEC_SUBSTITUTION = 1, MOESPEC_TRUNCATION = 2 } moespec_policy_t;
+/* Which experts compete for the shortlist.  FROM_ALL is Algorithm 1 as printed
+ * (all N experts ranked by s_i, so |S| = min(B, N)).  FROM_UNION restricts the
+ * candidates to the union E(D) of Eq. 3 (so |S| = min(B, |E|) and any
+ * B >= |E| reproduces the unbudgeted layer). */
+typedef enum { MOESPEC_FROM_ALL = 1, MOESPEC_FROM_UNION = 2 } moespec_shortlist_t;
+/* Expert-FFN kernel choice.  AUTO picks the tensor-core kernel for bf16 and the
+ * CUDA-core kernel for fp32 (fp32 accuracy needs full-precision FMAs). */
+typedef enum { MOESPEC_FFN_AUTO = 0, MOESPEC_FFN_CUDA_CORE = 1, MOESPEC_FFN_TENSOR_CORE = 2 } moespec_ffn_t;
+
+typedef struct {
+  int d;              /* model width; multiple of 64                                             */
+  int n_experts;      /* N, 1..256                                                               */
+  int f;              /* expert FFN width; multiple of 64 (128 for the tensor-core kernel)        */
+  int max_M;          /* largest M any call will pass (sizes the workspace), 1..4096              */
+  int max_k;          /* largest k any call will pass, 1..min(N, 32)                              */
+  int dtype;          /* moespec_dtype_t of weights and hidden; accumulation is always fp32       */
+  int out_dtype;      /* moespec_dtype_t of out; 0 = same as dtype.  MOESPEC_FP32 with bf16 weights
+                         returns the fp32 accumulators unrounded                                  */
+  int policy;         /* moespec_policy_t; 0 is invalid: the caller must choose                   */
+  int shortlist;      /* moespec_shortlist_t; 0 is invalid: the caller must choose                */
+  int renormalize;    /* 1: mixing weights are renormalised (Section 2.1, "OLMoE renormalizes"); 0: raw g_i */
+  int residual;       /* 1: out = hidden + MoE(hidden) rounded once to dtype; 0: out = MoE(hidden) */
+  int ffn_kernel;     /* moespec_ffn_t                                                            */
+  int device;         /* CUDA device ordinal                                                      */
+  const void *router_w;      /* device [N, d] row-major, dtype                                    */
+  const float *router_bias;  /* device [N] fp32, or NULL for the bias-free router of Eq. 1         */
+  const void *w_gate;        /* device [N, f, d], d contiguous, 16-byte aligned (W1 of SwiGLU)    */
+  const void *w_up;          /* device [N, f, d], d contiguous, 16-byte aligned (W3)              */
+  const void *w_down;        /* device [N, d, f], f contiguous, 16-byte aligned (W2)              */
+} moespec_layer_desc;
+
+typedef struct {
+  int n_union;        /* |E(D)|, Eq. 3                                                            */
+  int n_shortlist;    /* |S|                                                                      */
+  int n_active;       /* experts with at least one routed row (what is streamed from HBM)         */
+  int n_rows;         /* R = sum_t |A(t)| routed (token, expert) pairs                            */
+  int n_dropped;      /* M*k - R slots that received no expert                                    */
+  int status;         /* 0, MOESPEC_ERR_TIMEOUT or MOESPEC_ERR_INTERNAL from the last call        */
+  double coverage;    /* sum_{i in S} s_i / M, the routing mass kept by the shortlist (Section 4.6) */
+  long long weight_bytes; /* n_active * 3*d*f*sizeof(dtype): expert bytes the call had to read     */
+} moespec_stats;
+
+/* Create a layer (Section 2.1: router W_gate and N experts; k and renormalisation
+ * are properties of the architecture).  Validates the description, records the
+ * borrowed weight pointers, builds TMA descriptors and allocates the workspace
+ * for max_M tokens on desc->device.  *out_layer is written only on success.
+ * Errors: NULL_POINTER, INVALID_ARG, UNSUPPORTED, OUT_OF_MEMORY, CUDA. */
+int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_layer);
+
+/* Algorithm 1 for one layer.  hidden: device [M, d] row-major, dtype, 16-byte
+ * aligned.  out: device [M, d] in out_dtype, fully overwritten (exact zeros for a token with
+ * no kept expert when residual = 0).  out must not alias hidden.
+ * stream: a cudaStream_t (NULL = default stream).  Enqueues and returns.
+ * Errors: BAD_HANDLE, NULL_POINTER, INVALID_ARG, CUDA (launch failure). */
+int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int k, int B,
+                         void *out, void *stream);
+
+/* Same computation with HOST buffers: copies hidden (host [M, d]) to the device,
+ * runs the layer, copies the result into out (host [M, d], out_dtype) and synchronises the
+ * stream before returning.  Pinned host memory makes the copies asynchronous to
+ * other streams but is not required. */
+int moespec_verify_layer_host(moespec_layer_t *layer, const void *hidden_host, int M, int k, int B,
+                              void *out_host, void *stream);
+
+/* Steps after the router projection only (softmax, top-k, Eq. 5 scores,
+ * shortlist, Eq. 7 / Eq. 8 re-routing, Appendix C gather order), from caller-
+ * supplied fp32 logits: device [M, N] row-major.  Results stay in the workspace
+ * for moespec_get_routing.  This is the hook the integer half of the layer is
+ * checked through: fed the same fp32 logits, selection is exact. */
+int moespec_route_from_logits(moespec_layer_t *layer, const float *logits, int M, int k, int B,
+                              void *stream);
+
+/* Copy the routing state of the last verify/route call into HOST buffers (any
+ * may be NULL to skip it).  Synchronises the device.
+ *   S_rank[N]        shortlist in rank order (first *n_S entries valid)
+ *   topk_idx[M*k]    natural top-k per token, rank order
+ *   assign_idx[M*k]  kept expert per slot, -1 for a dropped slot.  Substitution
+ *                    fills slots 0..min(k,|S|)-1 in rank order; truncation keeps
+ *                    slot r of the natural top-k or drops it
+ *   gate_w[M*k]      mixing weight per slot (0 for a dropped slot)
+ *   count[N], offset[N+1]   rows per expert and their exclusive scan
+ *   perm_row2tok[R]  token index of each routed row; rows are ordered by
+ *                    (expert ascending, token ascending)
+ *   tokslot2row[M*k] row of each slot, -1 for a dropped slot
+ *   score[N]         fp64 s_i of Eq. 5
+ * M and k are those of the last call. */
+int moespec_get_routing(moespec_layer_t *layer, int *S_rank, int *n_S, int *topk_idx, int *assign_idx,
+                        float *gate_w, int *count, int *offset, int *perm_row2tok, int *tokslot2row,
+                        double *score, int *n_rows);
+
+/* Copy the fp32 router logits [M, N] of the last verify call to a HOST buffer.  Synchronises. */
+int moespec_get_logits(moespec_layer_t *layer, float *logits_host);
+
+/* Copy an intermediate of the last verify call to a HOST buffer of `bytes` bytes
+ * (clipped to the buffer's size in the workspace).  which: 0 = gathered rows
+ * x_perm [R, d] in dtype (Appendix C gather), 1 = h_mid [R, f] in dtype
+ * (silu(W1 x) * (W3 x) of the expert FFN), 2 = y [R, d] fp32 (expert outputs
+ * before the gate-weighted sum).  Rows follow perm_row2tok.  Synchronises. */
+int moespec_get_intermediate(moespec_layer_t *layer, int which, void *host_buf, long long bytes);
+
+/* Statistics of the last call.  Synchronises the device. */
+int moespec_get_stats(moespec_layer_t *layer, moespec_stats *stats);
+
+/* Per-kernel timing.  With profiling on, verify calls record a CUDA event on the
+ * stream before the first kernel and after every kernel (do not enable it while
+ * the stream is being captured into a graph).  get_kernel_times waits for the
+ * last verify call and writes the duration in milliseconds of each of its
+ * kernels, in launch order (router logits, routing, gather, expert FFN gate/up,
+ * expert FFN down, combine), into ms[0 .. min(capacity, *n_kernels)). */
+int moespec_set_profiling(moespec_layer_t *layer, int on);
+int moespec_get_kernel_times(moespec_layer_t *layer, float *ms, int capacity, int *n_kernels);
+
+/* Number of kernels the last verify call launched (host-side count). */
+int moespec_last_launch_count(moespec_layer_t *layer);
+
+/* Free the workspace and the handle.  NULL is accepted.  Borrowed buffers are untouched. */
+int moespec_destroy(moespec_layer_t *layer);
+
+const char *moespec_strerror(int status);
+/* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
+int moespec_last_cuda_error(void);
+int moespec_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOESPEC_H_ */

@@ -1,0 +1,446 @@
+// C ABI of libmoespec: handle life cycle, argument validation, workspace, launch order.
+#include "internal.h"
+
+#include <mutex>
+#include <new>
+#include <unordered_set>
+#include <vector>
+
+using namespace moespec;
+
+constexpr int kMaxProfiled = 8;   // kernels per verify call that can be bracketed by events
+
+struct moespec_layer {
+  unsigned long long magic;
+  moespec_layer_desc desc;
+  Workspace ws;
+  void *arena;
+  size_t arena_bytes;
+  int R_cap;
+  bool use_tc;
+  TcMaps maps;
+  int last_M, last_k;
+  int last_launches;
+  bool profiling;
+  cudaEvent_t ev[kMaxProfiled + 1];
+};
+
+namespace {
+
+constexpr unsigned long long kMagic = 0x4d6f455370656331ULL;
+thread_local int tl_cuda_error = 0;
+std::mutex g_mu;
+std::unordered_set<moespec_layer *> g_live;
+
+int cuda_fail(cudaError_t e) {
+  tl_cuda_error = (int)e;
+  return e == cudaErrorMemoryAllocation ? MOESPEC_ERR_OUT_OF_MEMORY : MOESPEC_ERR_CUDA;
+}
+
+bool is_live(moespec_layer *L) {
+  if (!L) return false;
+  std::lock_guard<std::mutex> lk(g_mu);
+  return g_live.count(L) != 0 && L->magic == kMagic;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool changed = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceGuard(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) {
+      err = cudaSetDevice(dev);
+      changed = err == cudaSuccess;
+    }
+  }
+  ~DeviceGuard() {
+    if (changed) cudaSetDevice(prev);
+  }
+};
+
+size_t elt_bytes(const moespec_layer_desc &d) { return d.dtype == MOESPEC_BF16 ? 2 : 4; }
+size_t out_elt_bytes(const moespec_layer_desc &d) { return (d.out_dtype ? d.out_dtype : d.dtype) == MOESPEC_BF16 ? 2 : 4; }
+
+struct Carver {
+  size_t off = 0;
+  char *base = nullptr;
+  template <typename T>
+  void take(T *&p, size_t count) {
+    off = (off + 255) & ~(size_t)255;
+    if (base) p = reinterpret_cast<T *>(base + off);
+    off += count * sizeof(T);
+  }
+  void take_bytes(void *&p, size_t bytes) {
+    off = (off + 255) & ~(size_t)255;
+    if (base) p = base + off;
+    off += bytes;
+  }
+};
+
+size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) {
+  Carver c;
+  c.base = base;
+  Workspace w{};
+  const size_t N = d.n_experts, M = d.max_M, K = d.max_k, eb = elt_bytes(d);
+  const size_t tiles_up = d.f / kTile + 1, tiles_down = d.d / kTile + 1;
+  // every expert can add at most one partial token chunk beyond the full ones
+  const size_t max_chunks = (size_t)R_cap / kMaxTokChunk + N;
+  c.take(w.logits, M * N);
+  c.take(w.prob, M * N);
+  c.take(w.score, N);
+  c.take(w.topk_idx, M * K);
+  c.take(w.S_rank, N);
+  c.take(w.assign_idx, M * K);
+  c.take(w.gate_w, M * K);
+  c.take(w.count, N);
+  c.take(w.offset, N + 1);
+  c.take(w.active, N);
+  c.take(w.perm_row2tok, (size_t)R_cap);
+  c.take(w.row2expert, (size_t)R_cap);
+  c.take(w.tokslot2row, M * K);
+  c.take(w.natmask, M * kMaskWords);
+  c.take(w.amask, M * kMaskWords);
+  c.take(w.units_up, max_chunks * tiles_up);
+  c.take(w.units_down, max_chunks * tiles_down);
+  c.take(w.counters, 16);
+  c.take(w.stats, 1);
+  c.take(w.status, 4);
+  c.take_bytes(w.x_perm, (size_t)R_cap * d.d * eb);
+  c.take_bytes(w.h_mid, (size_t)R_cap * d.f * eb);
+  c.take(w.y, (size_t)R_cap * d.d);
+  c.take_bytes(w.hidden_stage, M * d.d * eb);
+  c.take_bytes(w.out_stage, M * d.d * out_elt_bytes(d));
+  if (ws) *ws = w;
+  return (c.off + 255) & ~(size_t)255;
+}
+
+int validate_call(moespec_layer *L, int M, int k, int B) {
+  const moespec_layer_desc &d = L->desc;
+  if (M < 0 || M > d.max_M) return MOESPEC_ERR_INVALID_ARG;
+  if (k < 1 || k > d.max_k || k > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (B < 1) return MOESPEC_ERR_INVALID_ARG;
+  return MOESPEC_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
+  LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream};
+  int launches = 0, n = 0;
+  cudaError_t e;
+  // with profiling on, an event is recorded before the first kernel and after every kernel
+  auto mark = [&](int i) -> cudaError_t {
+    return (L->profiling && i <= kMaxProfiled) ? cudaEventRecord(L->ev[i], stream) : cudaSuccess;
+  };
+  if ((e = mark(0)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_router_logits(c, hidden)) != cudaSuccess) return cuda_fail(e);
+  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_route(c, L->ws.logits)) != cudaSuccess) return cuda_fail(e);
+  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
+  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  if (L->use_tc) {
+    for (int phase = 0; phase < 2; ++phase) {
+      if ((e = launch_ffn_tensor_core(c, &L->maps, phase)) != cudaSuccess) return cuda_fail(e);
+      if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+    }
+  } else {
+    for (int phase = 0; phase < 2; ++phase) {
+      if ((e = launch_ffn_cuda_core(c, phase)) != cudaSuccess) return cuda_fail(e);
+      if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+    }
+  }
+  if ((e = launch_combine(c, hidden, out)) != cudaSuccess) return cuda_fail(e);
+  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  (void)n;
+  L->last_M = M;
+  L->last_k = k;
+  L->last_launches = launches;
+  return MOESPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_layer) {
+  if (!desc || !out_layer) return MOESPEC_ERR_NULL_POINTER;
+  const moespec_layer_desc &d = *desc;
+  if (!d.router_w || !d.w_gate || !d.w_up || !d.w_down) return MOESPEC_ERR_NULL_POINTER;
+  if (d.dtype != MOESPEC_BF16 && d.dtype != MOESPEC_FP32) return MOESPEC_ERR_INVALID_ARG;
+  if (d.out_dtype != 0 && d.out_dtype != MOESPEC_BF16 && d.out_dtype != MOESPEC_FP32) return MOESPEC_ERR_INVALID_ARG;
+  if (d.dtype == MOESPEC_FP32 && d.out_dtype == MOESPEC_BF16) return MOESPEC_ERR_UNSUPPORTED;
+  if (d.policy != MOESPEC_SUBSTITUTION && d.policy != MOESPEC_TRUNCATION) return MOESPEC_ERR_INVALID_ARG;
+  if (d.shortlist != MOESPEC_FROM_ALL && d.shortlist != MOESPEC_FROM_UNION) return MOESPEC_ERR_INVALID_ARG;
+  if ((d.renormalize | 1) != 1 || (d.residual | 1) != 1) return MOESPEC_ERR_INVALID_ARG;
+  if (d.ffn_kernel < MOESPEC_FFN_AUTO || d.ffn_kernel > MOESPEC_FFN_TENSOR_CORE) return MOESPEC_ERR_INVALID_ARG;
+  if (d.d < 64 || d.f < 64 || d.n_experts < 1 || d.max_M < 1 || d.max_k < 1 || d.device < 0)
+    return MOESPEC_ERR_INVALID_ARG;
+  if (d.n_experts > kMaxExperts || d.max_k > kMaxK || d.max_k > d.n_experts || d.max_M > 4096 || d.d > 16384 ||
+      d.f > 65536)
+    return MOESPEC_ERR_INVALID_ARG;
+  if (d.d % 64 || d.f % 64) return MOESPEC_ERR_UNSUPPORTED;
+  if (!aligned16(d.router_w) || !aligned16(d.w_gate) || !aligned16(d.w_up) || !aligned16(d.w_down))
+    return MOESPEC_ERR_UNSUPPORTED;
+  bool use_tc = d.ffn_kernel == MOESPEC_FFN_TENSOR_CORE ||
+                (d.ffn_kernel == MOESPEC_FFN_AUTO && d.dtype == MOESPEC_BF16);
+  if (use_tc && (d.dtype != MOESPEC_BF16 || d.d % kTile || d.f % kTile)) {
+    if (d.ffn_kernel == MOESPEC_FFN_TENSOR_CORE) return MOESPEC_ERR_UNSUPPORTED;
+    use_tc = false;
+  }
+
+  int n_dev = 0;
+  cudaError_t e = cudaGetDeviceCount(&n_dev);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (d.device >= n_dev) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(d.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+
+  moespec_layer *L = new (std::nothrow) moespec_layer();
+  if (!L) return MOESPEC_ERR_OUT_OF_MEMORY;
+  L->magic = kMagic;
+  L->desc = d;
+  L->R_cap = d.max_M * d.max_k;
+  L->use_tc = use_tc;
+  L->arena_bytes = carve(d, L->R_cap, nullptr, nullptr);
+  e = cudaMalloc(&L->arena, L->arena_bytes);
+  if (e != cudaSuccess) {
+    delete L;
+    cudaGetLastError();
+    return cuda_fail(e);
+  }
+  e = cudaMemset(L->arena, 0, L->arena_bytes);
+  if (e != cudaSuccess) {
+    cudaFree(L->arena);
+    delete L;
+    return cuda_fail(e);
+  }
+  carve(d, L->R_cap, static_cast<char *>(L->arena), &L->ws);
+  if (use_tc) {
+    int cu_res = 0;
+    e = tc_encode_maps(d, L->ws, L->R_cap, &L->maps, &cu_res);
+    if (e == cudaSuccess) e = tc_configure();
+    if (e != cudaSuccess) {
+      cudaFree(L->arena);
+      delete L;
+      tl_cuda_error = cu_res ? cu_res : (int)e;
+      return MOESPEC_ERR_CUDA;
+    }
+  }
+  L->profiling = false;
+  for (int i = 0; i <= kMaxProfiled; ++i) {
+    e = cudaEventCreate(&L->ev[i]);
+    if (e != cudaSuccess) {
+      for (int j = 0; j < i; ++j) cudaEventDestroy(L->ev[j]);
+      cudaFree(L->arena);
+      delete L;
+      return cuda_fail(e);
+    }
+  }
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_live.insert(L);
+  }
+  *out_layer = L;
+  return MOESPEC_OK;
+}
+
+int moespec_verify_layer(moespec_layer_t *L, const void *hidden, int M, int k, int B, void *out, void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  int rc = validate_call(L, M, k, B);
+  if (rc) return rc;
+  if (M == 0) return MOESPEC_OK;
+  if (!hidden || !out) return MOESPEC_ERR_NULL_POINTER;
+  if (!aligned16(hidden) || !aligned16(out)) return MOESPEC_ERR_UNSUPPORTED;
+  if (hidden == out) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  return run_layer(L, hidden, M, k, B, out, static_cast<cudaStream_t>(stream));
+}
+
+int moespec_verify_layer_host(moespec_layer_t *L, const void *hidden_host, int M, int k, int B, void *out_host,
+                              void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  int rc = validate_call(L, M, k, B);
+  if (rc) return rc;
+  if (M == 0) return MOESPEC_OK;
+  if (!hidden_host || !out_host) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)M * L->desc.d * elt_bytes(L->desc);
+  cudaError_t e = cudaMemcpyAsync(L->ws.hidden_stage, hidden_host, bytes, cudaMemcpyHostToDevice, s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  rc = run_layer(L, L->ws.hidden_stage, M, k, B, L->ws.out_stage, s);
+  if (rc) return rc;
+  const size_t out_bytes = (size_t)M * L->desc.d * out_elt_bytes(L->desc);
+  e = cudaMemcpyAsync(out_host, L->ws.out_stage, out_bytes, cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return cuda_fail(e);
+  return MOESPEC_OK;
+}
+
+int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, int k, int B, void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  int rc = validate_call(L, M, k, B);
+  if (rc) return rc;
+  if (M == 0) return MOESPEC_OK;
+  if (!logits) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap,
+              static_cast<cudaStream_t>(stream)};
+  cudaError_t e = launch_route(c, logits);
+  if (e != cudaSuccess) return cuda_fail(e);
+  L->last_M = M;
+  L->last_k = k;
+  L->last_launches = 1;
+  return MOESPEC_OK;
+}
+
+#define MOESPEC_COPY_BACK(dst, src, count)                                                         \
+  do {                                                                                             \
+    if ((dst) && (count) > 0) {                                                                    \
+      cudaError_t e_ = cudaMemcpy((dst), (src), sizeof(*(dst)) * (size_t)(count), cudaMemcpyDeviceToHost); \
+      if (e_ != cudaSuccess) return cuda_fail(e_);                                                 \
+    }                                                                                              \
+  } while (0)
+
+int moespec_get_routing(moespec_layer_t *L, int *S_rank, int *n_S, int *topk_idx, int *assign_idx, float *gate_w,
+                        int *count, int *offset, int *perm_row2tok, int *tokslot2row, double *score,
+                        int *n_rows) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  int counters[8];
+  e = cudaMemcpy(counters, L->ws.counters, sizeof(counters), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  const int N = L->desc.n_experts, mk = L->last_M * L->last_k;
+  if (n_S) *n_S = counters[0];
+  if (n_rows) *n_rows = counters[2];
+  MOESPEC_COPY_BACK(S_rank, L->ws.S_rank, counters[0]);
+  MOESPEC_COPY_BACK(topk_idx, L->ws.topk_idx, mk);
+  MOESPEC_COPY_BACK(assign_idx, L->ws.assign_idx, mk);
+  MOESPEC_COPY_BACK(gate_w, L->ws.gate_w, mk);
+  MOESPEC_COPY_BACK(count, L->ws.count, N);
+  MOESPEC_COPY_BACK(offset, L->ws.offset, N + 1);
+  MOESPEC_COPY_BACK(perm_row2tok, L->ws.perm_row2tok, counters[2]);
+  MOESPEC_COPY_BACK(tokslot2row, L->ws.tokslot2row, mk);
+  MOESPEC_COPY_BACK(score, L->ws.score, N);
+  return MOESPEC_OK;
+}
+
+int moespec_get_logits(moespec_layer_t *L, float *logits_host) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!logits_host) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  MOESPEC_COPY_BACK(logits_host, L->ws.logits, L->last_M * L->desc.n_experts);
+  return MOESPEC_OK;
+}
+
+int moespec_get_intermediate(moespec_layer_t *L, int which, void *host_buf, long long bytes) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!host_buf) return MOESPEC_ERR_NULL_POINTER;
+  if (which < 0 || which > 2 || bytes < 0) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  const size_t eb = elt_bytes(L->desc), R = (size_t)L->R_cap;
+  const void *src = which == 0 ? L->ws.x_perm : which == 1 ? L->ws.h_mid : (const void *)L->ws.y;
+  size_t cap = which == 0 ? R * L->desc.d * eb : which == 1 ? R * L->desc.f * eb : R * L->desc.d * 4;
+  size_t n = (size_t)bytes < cap ? (size_t)bytes : cap;
+  if (n) {
+    e = cudaMemcpy(host_buf, src, n, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return MOESPEC_OK;
+}
+
+int moespec_get_stats(moespec_layer_t *L, moespec_stats *stats) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!stats) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  MOESPEC_COPY_BACK(stats, L->ws.stats, 1);
+  int status = 0;
+  e = cudaMemcpy(&status, L->ws.status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  stats->status = status;
+  return MOESPEC_OK;
+}
+
+int moespec_set_profiling(moespec_layer_t *L, int on) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  L->profiling = on != 0;
+  return MOESPEC_OK;
+}
+
+int moespec_get_kernel_times(moespec_layer_t *L, float *ms, int capacity, int *n_kernels) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!ms || !n_kernels) return MOESPEC_ERR_NULL_POINTER;
+  if (!L->profiling || L->last_launches <= 1) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  const int n = L->last_launches < kMaxProfiled ? L->last_launches : kMaxProfiled;
+  cudaError_t e = cudaEventSynchronize(L->ev[n]);
+  if (e != cudaSuccess) return cuda_fail(e);
+  *n_kernels = n;
+  for (int i = 0; i < n && i < capacity; ++i) {
+    e = cudaEventElapsedTime(&ms[i], L->ev[i], L->ev[i + 1]);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return MOESPEC_OK;
+}
+
+int moespec_last_launch_count(moespec_layer_t *L) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  return L->last_launches;
+}
+
+int moespec_destroy(moespec_layer_t *L) {
+  if (!L) return MOESPEC_OK;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (g_live.erase(L) == 0) return MOESPEC_ERR_BAD_HANDLE;
+  }
+  int rc = MOESPEC_OK;
+  {
+    DeviceGuard guard(L->desc.device);
+    for (int i = 0; i <= kMaxProfiled; ++i) cudaEventDestroy(L->ev[i]);
+    cudaError_t e = cudaFree(L->arena);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+  }
+  L->magic = 0;
+  delete L;
+  return rc;
+}
+
+const char *moespec_strerror(int status) {
+  switch (status) {
+    case MOESPEC_OK: return "ok";
+    case MOESPEC_ERR_INVALID_ARG: return "invalid argument";
+    case MOESPEC_ERR_NULL_POINTER: return "null pointer";
+    case MOESPEC_ERR_UNSUPPORTED: return "unsupported shape, dtype or alignment";
+    case MOESPEC_ERR_OUT_OF_MEMORY: return "out of device memory";
+    case MOESPEC_ERR_CUDA: return "CUDA call failed";
+    case MOESPEC_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case MOESPEC_ERR_INTERNAL: return "device-side consistency check failed";
+    case MOESPEC_ERR_BAD_HANDLE: return "bad or destroyed handle";
+    default: return "unknown status";
+  }
+}
+
+int moespec_last_cuda_error(void) { return tl_cuda_error; }
+int moespec_version(void) { return 100; }
+
+}  // extern "C"

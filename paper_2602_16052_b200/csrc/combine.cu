@@ -1,0 +1,76 @@
+// Gate-weighted combine: out_t = sum over the kept slots of wgt[t, slot] * y[row(t, slot)]
+// (outer sums of Eq. 2 / Eq. 7 / Eq. 8).  A token with no kept expert gets exact
+// zeros (Section 3.3).  Slots are added in a fixed order, so the result is
+// bitwise reproducible.  With the residual flag the layer input is added before
+// the single rounding to the storage dtype.
+#include "internal.h"
+
+namespace moespec {
+
+__device__ __forceinline__ float4 load4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ float4 load4(const __nv_bfloat16 *p) {
+  uint2 raw = *reinterpret_cast<const uint2 *>(p);
+  const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+  float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
+  return make_float4(a.x, a.y, b.x, b.y);
+}
+__device__ __forceinline__ void store4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 raw;
+  raw.x = *reinterpret_cast<uint32_t *>(&lo);
+  raw.y = *reinterpret_cast<uint32_t *>(&hi);
+  *reinterpret_cast<uint2 *>(p) = raw;
+}
+
+template <typename T, typename TO>
+__global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ y,
+                                                      const float *__restrict__ gate_w,
+                                                      const int *__restrict__ tokslot2row,
+                                                      const T *__restrict__ hidden, TO *__restrict__ out, int d,
+                                                      int k, int residual) {
+  const int t = blockIdx.x;
+  __shared__ int s_row[kMaxK];
+  __shared__ float s_w[kMaxK];
+  if (threadIdx.x < k) {
+    s_row[threadIdx.x] = tokslot2row[(size_t)t * k + threadIdx.x];
+    s_w[threadIdx.x] = gate_w[(size_t)t * k + threadIdx.x];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < k; ++s) {
+      const int row = s_row[s];
+      if (row < 0) continue;
+      const float w = s_w[s];
+      float4 v = load4(y + (size_t)row * d + c);
+      acc.x = fmaf(w, v.x, acc.x);
+      acc.y = fmaf(w, v.y, acc.y);
+      acc.z = fmaf(w, v.z, acc.z);
+      acc.w = fmaf(w, v.w, acc.w);
+    }
+    if (residual) {
+      float4 h = load4(hidden + (size_t)t * d + c);
+      acc.x += h.x; acc.y += h.y; acc.z += h.z; acc.w += h.w;
+    }
+    store4(out + (size_t)t * d + c, acc);
+  }
+}
+
+template <typename T, typename TO>
+static void launch_t(const LaunchCtx &c, const void *hidden, void *out) {
+  const moespec_layer_desc &D = *c.desc;
+  combine_kernel<T, TO><<<c.M, 256, 0, c.stream>>>(c.ws->y, c.ws->gate_w, c.ws->tokslot2row, (const T *)hidden,
+                                                   (TO *)out, D.d, c.k, D.residual);
+}
+
+cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out) {
+  const moespec_layer_desc &D = *c.desc;
+  const int od = D.out_dtype ? D.out_dtype : D.dtype;
+  if (D.dtype == MOESPEC_BF16 && od == MOESPEC_BF16) launch_t<__nv_bfloat16, __nv_bfloat16>(c, hidden, out);
+  else if (D.dtype == MOESPEC_BF16) launch_t<__nv_bfloat16, float>(c, hidden, out);
+  else launch_t<float, float>(c, hidden, out);
+  return cudaGetLastError();
+}
+
+}  // namespace moespec

@@ -1,0 +1,395 @@
+// Tensor-core expert FFN for bf16: the weight-streaming kernel of the layer.
+//
+// Work unit = one 128-row slab of one kept expert's weight matrix against one
+// chunk (<= 256) of that expert's routed rows.  Weights are the MMA A operand
+// (rows of W on the M axis, so every weight byte is read from HBM exactly once),
+// routed token rows are the B operand (N axis, padded to a multiple of 32),
+// fp32 accumulators live in tensor memory.
+//
+//   phase 0 (gate/up):  D_g = W1[e, slab, :] X_e^T,  D_u = W3[e, slab, :] X_e^T,
+//                       h_mid[row, slab] = bf16(silu(D_g) * D_u)
+//   phase 1 (down):     D = W2[e, slab, :] H_e^T,     y[row, slab] = D  (fp32)
+//
+// One persistent CTA per SM, six warps:
+//   warp 0  lane 0: TMA producer.  Streams 64-wide K chunks of the weight slab(s)
+//                   (3-D tensor map, expert id is the outer coordinate: no
+//                   stacking copy) and of the token rows into a ring of stages.
+//   warp 1  lane 0: issues tcgen05.mma (kind::f16, M=128, N=n_pad, K=16) from the
+//                   stage's swizzled shared memory into TMEM; tcgen05.commit frees
+//                   the stage and finally publishes the accumulator.
+//   warps 2-5     : epilogue.  tcgen05.ld the accumulator (one TMEM lane quarter
+//                   per warp), apply SwiGLU, store to global.
+// Every wait is bounded: on expiry the CTA raises an abort flag, records
+// MOESPEC_ERR_TIMEOUT in the status word, drains its own copies, frees TMEM and
+// returns.
+#include "internal.h"
+
+namespace moespec {
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kChunkK = 64;                      // bf16 elements per 128-byte swizzle row
+constexpr int kABytes = kTile * kChunkK * 2;     // 16 KB: one weight slab chunk
+constexpr int kBOffset = 2 * kABytes;            // token rows start after two weight chunks
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 227 * 1024;
+constexpr int kCtrlBytes = 256;                  // barriers + TMEM base + abort flag
+constexpr uint32_t kTmemCols = 512;
+constexpr long long kSpinLimitCycles = 2000000000LL;   // ~1 s at 2 GHz
+
+struct TcArgs {
+  const Unit *units;
+  const int *n_units;
+  int phase;            // 0 gate/up, 1 down
+  int k_chunks;         // K / 64
+  int n_stages;
+  int stage_bytes;
+  int acc_bufs;         // 1 or 2 accumulator buffers of 256 TMEM columns
+  void *out;            // h_mid (bf16) or y (fp32)
+  int out_ld;           // f or d
+  int *status;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting or the limit expired.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try(bar, parity)) return true;
+    if ((i & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > kSpinLimitCycles) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows at a
+// 128-byte pitch, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);         // start address
+  d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                          // descriptor version
+  d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+}
+
+}  // namespace
+
+__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // stages first (1024-byte aligned for the 128-byte swizzle), control block after
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t ctrl = smem_base + (uint32_t)a.n_stages * (uint32_t)a.stage_bytes;
+  uint8_t *ctrl_gen = smem_gen + (size_t)a.n_stages * a.stage_bytes;
+  const uint32_t bar_full = ctrl;                       // [kMaxStages]
+  const uint32_t bar_empty = ctrl + 8 * kMaxStages;     // [kMaxStages]
+  const uint32_t bar_acc_full = ctrl + 16 * kMaxStages; // [2]
+  const uint32_t bar_acc_empty = bar_acc_full + 16;     // [2]
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 32);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + 16 * kMaxStages + 36);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_units = *a.n_units;
+  const int n_stages = a.n_stages;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(bar_full + 8 * s, 1);
+      mbar_init(bar_empty + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_acc_full + 8 * b, 1);
+      mbar_init(bar_acc_empty + 8 * b, 128);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                     smem_u32(const_cast<uint32_t *>(tmem_slot))),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const CUtensorMap *map_a0 = a.phase == 0 ? &maps.w_gate : &maps.w_down;
+  const CUtensorMap *map_a1 = &maps.w_up;
+  const CUtensorMap *map_b = a.phase == 0 ? &maps.x_perm : &maps.h_mid;
+  const uint32_t a_bytes = a.phase == 0 ? 2u * kABytes : (uint32_t)kABytes;
+
+  if (warp == 0 && lane == 0) {
+    // ===================================================== TMA producer
+    uint32_t it = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      const Unit un = a.units[u];
+      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      for (int kc = 0; kc < a.k_chunks; ++kc, ++it) {
+        const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
+        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t full = bar_full + 8 * s;
+        const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
+        mbar_expect_tx(full, a_bytes + (uint32_t)n_pad * 128u);
+        tma_load_3d(stage, map_a0, full, kc * kChunkK, un.tile * kTile, un.expert);
+        if (a.phase == 0) tma_load_3d(stage + kABytes, map_a1, full, kc * kChunkK, un.tile * kTile, un.expert);
+        for (int b = 0; b < n_pad / kTokBox; ++b)
+          tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
+      }
+    }
+    if (!ok) {
+      // drain: wait (bounded) until every copy this thread issued has landed
+      const uint32_t lo = it > (uint32_t)n_stages ? it - n_stages : 0u;
+      for (uint32_t j = lo; j < it; ++j) {
+        const long long t0 = clock64();
+        while (!mbar_try(bar_full + 8 * (j % n_stages), (j / n_stages) & 1u))
+          if (clock64() - t0 > kSpinLimitCycles) break;
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ===================================================== MMA issuer
+    uint32_t it = 0, acc_it = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
+      const Unit un = a.units[u];
+      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const uint32_t idesc = instr_desc_bf16(n_pad);
+      const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
+      if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t tmem_d = tmem_base + ab * 256u;
+      for (int kc = 0; kc < a.k_chunks; ++kc, ++it) {
+        const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
+        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
+#pragma unroll
+        for (int kk = 0; kk < kChunkK / 16; ++kk) {
+          const uint32_t acc = (kc > 0 || kk > 0) ? 1u : 0u;
+          const uint64_t bdesc = smem_desc_sw128(stage + kBOffset + kk * 32);
+          tc_mma_bf16(tmem_d, smem_desc_sw128(stage + kk * 32), bdesc, idesc, acc);
+          if (a.phase == 0)
+            tc_mma_bf16(tmem_d + (uint32_t)n_pad, smem_desc_sw128(stage + kABytes + kk * 32), bdesc, idesc, acc);
+        }
+        tc_commit(bar_empty + 8 * s);      // stage reusable once these MMAs have read it
+      }
+      if (ok) tc_commit(bar_acc_full + 8 * ab);
+    }
+  } else if (warp >= 2) {
+    // ===================================================== epilogue
+    const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 belong to this warp
+    const int row_in_tile = quarter * 32 + lane;
+    uint32_t acc_it = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
+      const Unit un = a.units[u];
+      const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
+      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
+      const int col_out = un.tile * kTile + row_in_tile;    // index along f (phase 0) or d (phase 1)
+      for (int c0 = 0; c0 < un.n_rows; c0 += 16) {
+        uint32_t g[16];
+        tc_ld16(taddr + c0, g);
+        if (a.phase == 0) {
+          uint32_t up[16];
+          tc_ld16(taddr + n_pad + c0, up);
+          tc_ld_wait();
+          __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            if (c0 + i < un.n_rows) {
+              const float gv = __uint_as_float(g[i]), uv = __uint_as_float(up[i]);
+              const float m = gv / (1.f + __expf(-gv)) * uv;
+              out[(size_t)(un.row0 + c0 + i) * a.out_ld + col_out] = __float2bfloat16_rn(m);
+            }
+          }
+        } else {
+          tc_ld_wait();
+          float *out = reinterpret_cast<float *>(a.out);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (c0 + i < un.n_rows) out[(size_t)(un.row0 + c0 + i) * a.out_ld + col_out] = __uint_as_float(g[i]);
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(bar_acc_empty + 8 * ab);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, (int)MOESPEC_ERR_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static cudaError_t get_encode_fn(EncodeTiledFn *fn) {
+  void *p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
+  if (e != cudaSuccess) return e;
+  if (q != cudaDriverEntryPointSuccess || !p) return cudaErrorNotSupported;
+  *fn = reinterpret_cast<EncodeTiledFn>(p);
+  return cudaSuccess;
+}
+
+cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps, int *cu_result) {
+  EncodeTiledFn enc = nullptr;
+  cudaError_t e = get_encode_fn(&enc);
+  if (e != cudaSuccess) return e;
+  const cuuint32_t ones[3] = {1, 1, 1};
+  auto weights = [&](CUtensorMap *m, const void *base, int rows, int K) -> CUresult {
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)d.n_experts};
+    cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)rows * K * 2};
+    cuuint32_t box[3] = {kChunkK, kTile, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, ones,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  };
+  auto rows2d = [&](CUtensorMap *m, void *base, int K) -> CUresult {
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)R_cap};
+    cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    cuuint32_t box[2] = {kChunkK, kTokBox};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  };
+  CUresult r;
+  if ((r = weights(&maps->w_gate, d.w_gate, d.f, d.d)) != CUDA_SUCCESS ||
+      (r = weights(&maps->w_up, d.w_up, d.f, d.d)) != CUDA_SUCCESS ||
+      (r = weights(&maps->w_down, d.w_down, d.d, d.f)) != CUDA_SUCCESS ||
+      (r = rows2d(&maps->x_perm, ws.x_perm, d.d)) != CUDA_SUCCESS ||
+      (r = rows2d(&maps->h_mid, ws.h_mid, d.f)) != CUDA_SUCCESS) {
+    *cu_result = (int)r;
+    return cudaErrorInvalidValue;
+  }
+  return cudaSuccess;
+}
+
+cudaError_t tc_configure() {
+  return cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
+}
+
+static int sm_count_cached(int device) {
+  static int cached[64] = {0};
+  if (device < 64 && cached[device]) return cached[device];
+  int n = 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 148;
+  if (device < 64) cached[device] = n;
+  return n;
+}
+
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, int phase) {
+  const moespec_layer_desc &D = *c.desc;
+  const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
+  TcArgs a;
+  a.stage_bytes = kBOffset + n_pad_max * 128;
+  int stages = (kSmemBudget - 1024 - kCtrlBytes) / a.stage_bytes;
+  a.n_stages = stages > kMaxStages ? kMaxStages : stages;
+  a.acc_bufs = 2 * n_pad_max <= 256 ? 2 : 1;
+  a.status = c.ws->status;
+  const int grid = sm_count_cached(D.device);
+  const size_t smem = (size_t)a.n_stages * a.stage_bytes + 1024 + kCtrlBytes;
+  a.phase = phase;
+  if (phase == 0) {
+    a.units = c.ws->units_up;
+    a.n_units = c.ws->counters + 3;
+    a.k_chunks = D.d / kChunkK;
+    a.out = c.ws->h_mid;
+    a.out_ld = D.f;
+  } else {
+    a.units = c.ws->units_down;
+    a.n_units = c.ws->counters + 4;
+    a.k_chunks = D.f / kChunkK;
+    a.out = c.ws->y;
+    a.out_ld = D.d;
+  }
+  ffn_tc_kernel<<<grid, kThreads, smem, c.stream>>>(*maps, a);
+  return cudaGetLastError();
+}
+
+}  // namespace moespec

@@ -1,0 +1,81 @@
+// Internal declarations shared by the translation units of libmoespec.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "../../include/moespec.h"
+
+namespace moespec {
+
+constexpr int kMaxExperts = 256;           // N limit: 8 experts per lane in the warp-wide rankings
+constexpr int kMaskWords = kMaxExperts / 32;
+constexpr int kMaxK = 32;
+constexpr int kTile = 128;                 // weight rows per tensor-core work unit (MMA M)
+constexpr int kTokBox = 32;                // token rows per TMA box of the B operand
+constexpr int kMaxTokChunk = 256;          // tokens per work unit (MMA N limit)
+
+// One tensor-core work unit: a 128-row slab of one expert's weight matrix
+// against one chunk (<= 256) of that expert's routed rows.
+struct Unit {
+  int expert;
+  int tile;       // slab index along f (gate/up phase) or d (down phase)
+  int row0;       // first routed row of the chunk
+  int n_rows;     // rows in the chunk (1..256)
+};
+
+// Device-resident routing state and scratch of one layer handle.
+struct Workspace {
+  float *logits;        // [max_M, N]
+  double *prob;         // [max_M, N]
+  double *score;        // [N]
+  int *topk_idx;        // [max_M, max_k]
+  int *S_rank;          // [N]
+  int *assign_idx;      // [max_M, max_k]
+  float *gate_w;        // [max_M, max_k]
+  int *count;           // [N]
+  int *offset;          // [N+1]
+  int *active;          // [N]
+  int *perm_row2tok;    // [R_cap]
+  int *row2expert;      // [R_cap]
+  int *tokslot2row;     // [max_M, max_k]
+  unsigned *natmask;    // [max_M, 8] bit i of row t: expert i in T_k(h_t)
+  unsigned *amask;      // [max_M, 8] bit i of row t: expert i in A(t)
+  Unit *units_up;       // gate/up units
+  Unit *units_down;     // down units
+  int *counters;        // [0]=n_S [1]=n_active [2]=R [3]=n_units_up [4]=n_units_down
+  moespec_stats *stats; // device copy
+  int *status;          // device status word (0 = ok)
+  void *x_perm;         // [R_cap, d] dtype
+  void *h_mid;          // [R_cap, f] dtype
+  float *y;             // [R_cap, d] fp32
+  void *hidden_stage;   // [max_M, d] dtype (host-buffer variant)
+  void *out_stage;      // [max_M, d] dtype
+};
+
+struct LaunchCtx {
+  const moespec_layer_desc *desc;
+  const Workspace *ws;
+  int M, k, B;
+  int R_cap;            // max_M * max_k
+  cudaStream_t stream;
+};
+
+// routing.cu
+cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden);
+cudaError_t launch_route(const LaunchCtx &c, const float *logits);
+cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
+// ffn_simple.cu
+cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down
+// ffn_tc.cu
+struct TcMaps {
+  CUtensorMap w_gate, w_up, w_down, x_perm, h_mid;
+};
+cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
+                           int *cu_result);
+cudaError_t tc_configure();   // one-time function attributes
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, int phase);   // 0 gate/up, 1 down
+// combine.cu
+cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out);
+
+}  // namespace moespec

@@ -1,0 +1,238 @@
+"""Thin ctypes binding over libmoespec.so (argument marshalling only).
+
+Names mirror the C ABI in include/moespec.h.  Every step of the layer runs in
+the library's CUDA kernels; nothing here computes.  Importing this module
+loads the library and raises if it has not been built: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmoespec.so")
+
+BF16, FP32 = 1, 2
+SUBSTITUTION, TRUNCATION = 1, 2
+FROM_ALL, FROM_UNION = 1, 2
+FFN_AUTO, FFN_CUDA_CORE, FFN_TENSOR_CORE = 0, 1, 2
+
+OK = 0
+ERR_INVALID_ARG, ERR_NULL_POINTER, ERR_UNSUPPORTED, ERR_OUT_OF_MEMORY = -1, -2, -3, -4
+ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL, ERR_BAD_HANDLE = -5, -6, -7, -8
+
+EXPORTS = [
+    "moespec_layer_create", "moespec_verify_layer", "moespec_verify_layer_host",
+    "moespec_route_from_logits", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
+    "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
+    "moespec_version",
+]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [
+        ("d", C.c_int), ("n_experts", C.c_int), ("f", C.c_int), ("max_M", C.c_int), ("max_k", C.c_int),
+        ("dtype", C.c_int), ("out_dtype", C.c_int), ("policy", C.c_int), ("shortlist", C.c_int), ("renormalize", C.c_int),
+        ("residual", C.c_int), ("ffn_kernel", C.c_int), ("device", C.c_int),
+        ("router_w", C.c_void_p), ("router_bias", C.c_void_p),
+        ("w_gate", C.c_void_p), ("w_up", C.c_void_p), ("w_down", C.c_void_p),
+    ]
+
+
+class Stats(C.Structure):
+    _fields_ = [
+        ("n_union", C.c_int), ("n_shortlist", C.c_int), ("n_active", C.c_int), ("n_rows", C.c_int),
+        ("n_dropped", C.c_int), ("status", C.c_int), ("coverage", C.c_double), ("weight_bytes", C.c_longlong),
+    ]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_}
+
+
+class MoeSpecError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().moespec_strerror(code).decode()
+        cuda = lib().moespec_last_cuda_error() if code == ERR_CUDA else 0
+        super().__init__(f"{where}: {msg} ({code})" + (f", cudaError {cuda}" if cuda else ""))
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the library once.  Raises if it is missing: the layer has no other implementation."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is not built; run python -m paper_2602_16052_b200.build")
+        L = C.CDLL(LIB_PATH)
+        vp, ci = C.c_void_p, C.c_int
+        L.moespec_layer_create.argtypes = [C.POINTER(LayerDesc), C.POINTER(vp)]
+        L.moespec_verify_layer.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.moespec_verify_layer_host.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.moespec_route_from_logits.argtypes = [vp, vp, ci, ci, ci, vp]
+        L.moespec_get_routing.argtypes = [vp] + [vp] * 11
+        L.moespec_get_logits.argtypes = [vp, vp]
+        L.moespec_get_intermediate.argtypes = [vp, ci, vp, C.c_longlong]
+        L.moespec_get_stats.argtypes = [vp, C.POINTER(Stats)]
+        L.moespec_set_profiling.argtypes = [vp, ci]
+        L.moespec_get_kernel_times.argtypes = [vp, vp, ci, vp]
+        L.moespec_last_launch_count.argtypes = [vp]
+        L.moespec_destroy.argtypes = [vp]
+        L.moespec_strerror.argtypes = [ci]
+        L.moespec_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if getattr(L, name).restype is not C.c_char_p:
+                getattr(L, name).restype = ci
+        _lib = L
+    return _lib
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise MoeSpecError(code, where)
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+class Layer:
+    """One MoE layer handle: moespec_layer_create / moespec_verify_layer / moespec_destroy.
+
+    Weight tensors are borrowed; this object keeps references so they outlive the handle.
+    """
+
+    def __init__(self, router_w, router_bias, w_gate, w_up, w_down, *, max_M: int, max_k: int,
+                 policy: int = SUBSTITUTION, shortlist: int = FROM_ALL, renormalize: bool = True,
+                 residual: bool = False, ffn_kernel: int = FFN_AUTO, out_dtype: Optional[torch.dtype] = None):
+        for t in (router_w, w_gate, w_up, w_down):
+            if not (t.is_cuda and t.is_contiguous()):
+                raise ValueError("weights must be contiguous CUDA tensors")
+        N, d = router_w.shape
+        f = w_gate.shape[1]
+        if tuple(w_gate.shape) != (N, f, d) or tuple(w_up.shape) != (N, f, d) or tuple(w_down.shape) != (N, d, f):
+            raise ValueError("weight shapes must be [N,f,d], [N,f,d], [N,d,f]")
+        dt = {torch.bfloat16: BF16, torch.float32: FP32}[router_w.dtype]
+        if router_bias is not None:
+            router_bias = router_bias.to(device=router_w.device, dtype=torch.float32).contiguous()
+        self._keep = (router_w, router_bias, w_gate, w_up, w_down)
+        self.d, self.N, self.f, self.max_M, self.max_k = d, N, f, max_M, max_k
+        self.dtype = router_w.dtype
+        self.out_dtype = out_dtype or router_w.dtype
+        self.device = router_w.device
+        desc = LayerDesc(d=d, n_experts=N, f=f, max_M=max_M, max_k=max_k, dtype=dt,
+                         out_dtype={torch.bfloat16: BF16, torch.float32: FP32}[self.out_dtype], policy=policy,
+                         shortlist=shortlist, renormalize=int(renormalize), residual=int(residual),
+                         ffn_kernel=ffn_kernel, device=router_w.device.index or 0,
+                         router_w=router_w.data_ptr(),
+                         router_bias=None if router_bias is None else router_bias.data_ptr(),
+                         w_gate=w_gate.data_ptr(), w_up=w_up.data_ptr(), w_down=w_down.data_ptr())
+        h = C.c_void_p()
+        _check(lib().moespec_layer_create(C.byref(desc), C.byref(h)), "moespec_layer_create")
+        self._h = h
+        self._last = (0, 0)
+
+    # -- the hot path
+    def verify_layer(self, hidden: torch.Tensor, k: int, B: int, out: Optional[torch.Tensor] = None, stream=None):
+        M = hidden.shape[0]
+        if out is None:
+            out = torch.empty(hidden.shape, dtype=self.out_dtype, device=hidden.device)
+        _check(lib().moespec_verify_layer(self._h, hidden.data_ptr(), M, k, B, out.data_ptr(), _stream_ptr(stream)),
+               "moespec_verify_layer")
+        self._last = (M, k)
+        return out
+
+    def verify_layer_host(self, hidden_host: torch.Tensor, k: int, B: int, out_host: torch.Tensor, stream=None):
+        M = hidden_host.shape[0]
+        _check(lib().moespec_verify_layer_host(self._h, hidden_host.data_ptr(), M, k, B, out_host.data_ptr(),
+                                               _stream_ptr(stream)), "moespec_verify_layer_host")
+        self._last = (M, k)
+        return out_host
+
+    def route_from_logits(self, logits: torch.Tensor, k: int, B: int, stream=None):
+        M = logits.shape[0]
+        assert logits.dtype == torch.float32 and logits.is_cuda and logits.is_contiguous()
+        _check(lib().moespec_route_from_logits(self._h, logits.data_ptr(), M, k, B, _stream_ptr(stream)),
+               "moespec_route_from_logits")
+        self._last = (M, k)
+
+    # -- introspection
+    def get_routing(self) -> dict:
+        M, k = self._last
+        N = self.N
+        i32 = lambda n: np.full(max(n, 1), -7, dtype=np.int32)
+        S, nS, nR = i32(N), C.c_int(0), C.c_int(0)
+        topk, assign, slot2row = i32(M * k), i32(M * k), i32(M * k)
+        gate = np.zeros(max(M * k, 1), dtype=np.float32)
+        count, offset = i32(N), i32(N + 1)
+        perm = i32(M * k)
+        score = np.zeros(N, dtype=np.float64)
+        _check(lib().moespec_get_routing(self._h, _np_ptr(S), C.cast(C.byref(nS), C.c_void_p), _np_ptr(topk),
+                                         _np_ptr(assign), _np_ptr(gate), _np_ptr(count), _np_ptr(offset),
+                                         _np_ptr(perm), _np_ptr(slot2row), _np_ptr(score),
+                                         C.cast(C.byref(nR), C.c_void_p)), "moespec_get_routing")
+        R = nR.value
+        return {"S": S[:nS.value].tolist(), "topk_idx": topk[:M * k].reshape(M, k),
+                "assign_idx": assign[:M * k].reshape(M, k), "gate_w": gate[:M * k].reshape(M, k),
+                "count": count.tolist(), "offset": offset.tolist(), "perm_row2tok": perm[:R].tolist(),
+                "tokslot2row": slot2row[:M * k].reshape(M, k), "score": score, "n_rows": R}
+
+    def get_logits(self) -> np.ndarray:
+        M, _ = self._last
+        z = np.zeros((M, self.N), dtype=np.float32)
+        _check(lib().moespec_get_logits(self._h, _np_ptr(z)), "moespec_get_logits")
+        return z
+
+    def get_intermediate(self, which: str, n_rows: int) -> torch.Tensor:
+        """Host copy of x_perm [R,d], h_mid [R,f] (layer dtype) or y [R,d] (fp32) of the last call."""
+        idx = {"x_perm": 0, "h_mid": 1, "y": 2}[which]
+        cols = self.f if idx == 1 else self.d
+        t = torch.empty((n_rows, cols), dtype=torch.float32 if idx == 2 else self.dtype)
+        if n_rows:
+            _check(lib().moespec_get_intermediate(self._h, idx, t.data_ptr(), t.numel() * t.element_size()),
+                   "moespec_get_intermediate")
+        return t
+
+    def get_stats(self) -> dict:
+        st = Stats()
+        _check(lib().moespec_get_stats(self._h, C.byref(st)), "moespec_get_stats")
+        return st.as_dict()
+
+    KERNEL_NAMES = ("router_logits", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
+
+    def set_profiling(self, on: bool):
+        _check(lib().moespec_set_profiling(self._h, int(on)), "moespec_set_profiling")
+
+    def get_kernel_times(self) -> dict:
+        """Milliseconds per kernel of the last verify call (profiling must be on)."""
+        ms = (C.c_float * 8)()
+        n = C.c_int(0)
+        _check(lib().moespec_get_kernel_times(self._h, C.cast(ms, C.c_void_p), 8, C.cast(C.byref(n), C.c_void_p)),
+               "moespec_get_kernel_times")
+        return {self.KERNEL_NAMES[i]: float(ms[i]) for i in range(min(n.value, len(self.KERNEL_NAMES)))}
+
+    def last_launch_count(self) -> int:
+        return lib().moespec_last_launch_count(self._h)
+
+    def destroy(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            code = lib().moespec_destroy(self._h)
+            self._h = None
+            _check(code, "moespec_destroy")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

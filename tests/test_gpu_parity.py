@@ -1,0 +1,291 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on seeded synthetic inputs.
+
+Integer work (shortlist, assignment, gather order) is compared bit for bit given
+the oracle's fp32 logits; layer outputs within the stated floating-point bar:
+max |err| <= 2e-2 * RMS(reference) for bf16 weights with fp32 accumulation, and
+max |err| <= 1e-5 * max(|ref|, RMS(ref)) per element for the fp32 configuration.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moespec_oracle as orc
+from paper_2602_16052_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+BF16_TOL = 2e-2
+FP32_TOL = 1e-5
+
+
+def ms():
+    from paper_2602_16052_b200 import moespec
+    return moespec
+
+
+def make_layer(case, max_M, max_k, **kw):
+    return ms().Layer(case["router_w"], case["router_bias"], case["w_gate"], case["w_up"], case["w_down"],
+                      max_M=max_M, max_k=max_k, **kw)
+
+
+def check_out(out, ref, dtype):
+    o = out.to("cpu", torch.float64).numpy()
+    # RMS over the tokens that received an expert: rows the policy zeroed (Section 3.3) must be exact zeros and
+    # would otherwise deflate the scale the tolerance is stated against
+    live = np.any(ref != 0.0, axis=1)
+    assert not np.any(o[~live]), "a token with no kept expert must get exact zeros"
+    rms = float(np.sqrt(np.mean(ref[live] ** 2))) if live.any() else 0.0
+    if dtype == "bf16" and out.dtype == torch.float32:
+        err = float(np.max(np.abs(o - ref)))
+        assert err <= BF16_TOL * rms, f"max err {err:.3e} > {BF16_TOL} * rms {rms:.3e}"
+    elif dtype == "bf16":
+        # out stored as bf16: the stated bar plus the final rounding of the result itself (half an ulp <= 2^-9 |ref|)
+        bound = BF16_TOL * rms + 2.0 ** -9 * np.abs(ref)
+        assert np.all(np.abs(o - ref) <= bound), f"worst {np.max(np.abs(o - ref) / np.maximum(bound, 1e-300)):.2f}x of bound"
+    else:
+        bound = FP32_TOL * np.maximum(np.abs(ref), rms)
+        bad = np.abs(o - ref) > bound
+        assert not bad.any(), f"{bad.sum()} elements beyond 1e-5 relative; worst {np.max(np.abs(o - ref) / bound):.2f}x"
+
+
+def run_e2e(cfg, M, B, policy, mode, renorm, ffn_kernel, seed=0, k=None, case=None, layer=None, residual=False,
+            out_dtype=torch.float32):
+    """Run the GPU layer, then the oracle on the GPU's own fp32 logits; also check the logits."""
+    k = cfg.k if k is None else k
+    case = case or H.make_case(cfg, M, seed)
+    own = layer is None
+    layer = layer or make_layer(case, max_M=max(M, 1), max_k=k, policy=policy, shortlist=mode,
+                                renormalize=renorm, ffn_kernel=ffn_kernel, residual=residual, out_dtype=out_dtype)
+    out = layer.verify_layer(case["hidden"], k, B)
+    torch.cuda.synchronize()
+    st = layer.get_stats()
+    assert st["status"] == 0
+    z_gpu = layer.get_logits()
+    z_ref = orc.router_logits(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]))
+    zerr = 3e-6 if cfg.dtype == "fp32" else 2e-5
+    assert np.max(np.abs(z_gpu.astype(np.float64) - z_ref)) <= zerr * max(1.0, np.abs(z_ref).max())
+    r = H.oracle_run(case, k, B, policy, mode, renorm, logits=z_gpu)
+    H.compare_routing(layer.get_routing(), r, policy, k)
+    ref = r["out"] + (H.f64(case["hidden"]) if residual else 0.0)
+    check_out(out, ref, cfg.dtype)
+    assert st["n_union"] == len(r["union"]) and st["n_shortlist"] == len(r["S"])
+    assert st["n_active"] == len(r["active"]) and st["n_rows"] == len(r["perm_row2tok"])
+    assert st["n_dropped"] == M * k - st["n_rows"]
+    assert abs(st["coverage"] - r["coverage"]) < 1e-12
+    assert st["weight_bytes"] == len(r["active"]) * cfg.expert_weight_bytes()
+    # the oracle on its own logits makes the same selection unless a near-tie sits inside the logit error
+    r_own = H.oracle_route(z_ref, k, B, policy, mode, renorm)
+    if r_own["S"] != r["S"] or r_own["assign"] != r["assign"]:
+        zgap, sgap = H.selection_margins(r_own, min(k, cfg.n_experts), None if mode == orc.FROM_ALL else r_own["union"])
+        assert min(zgap, sgap) < 1e-4, "selection differs from the oracle's without a certified near-tie"
+    if own:
+        layer.destroy()
+    return out, r, st
+
+
+# ------------------------------------------------------------------ generator
+def test_generator_is_bit_identical_on_gpu():
+    cfg = synth.CONFIGS["olmoe"].with_(f=128, n_experts=4)
+    for a, b in zip(synth.gen_expert_weights(cfg, 3, 1, "cpu"), synth.gen_expert_weights(cfg, 3, 1, "cuda")):
+        assert torch.equal(a, b.cpu())
+    assert torch.equal(synth.gen_hidden(cfg, 33, 5, 2, "cpu"), synth.gen_hidden(cfg, 33, 5, 2, "cuda").cpu())
+    tiny = synth.CONFIGS["tiny"]
+    assert torch.equal(synth.gen_hidden(tiny, 15, 0, 0, "cpu"), synth.gen_hidden(tiny, 15, 0, 0, "cuda").cpu())
+    wc, bc = synth.gen_router(cfg, 1, 0, "cpu")
+    wg, bg = synth.gen_router(cfg, 1, 0, "cuda")
+    assert torch.equal(wc, wg.cpu()) and torch.equal(bc, bg.cpu())
+
+
+# ------------------------------------------------------------------ integer half, bit exact
+ROUTE_SHAPES = [
+    ("tiny", dict(), [1, 15], [1, 2, 4, 8, 16, 40]),
+    ("olmoe", dict(f=128), [1, 7, 63, 127, 255], [8, 16, 32, 48, 64]),
+    ("qwen3", dict(f=128), [63, 127], [4, 32, 64, 128]),
+    ("mixtral", dict(f=128, d=512), [15, 63], [1, 2, 4, 6, 8]),
+]
+
+
+@pytest.mark.parametrize("name,shrink,Ms,Bs", ROUTE_SHAPES)
+def test_routing_bit_exact_from_oracle_logits(name, shrink, Ms, Bs):
+    cfg = synth.CONFIGS[name].with_(**shrink)
+    for M in Ms:
+        case = H.make_case(cfg, M, seed=11)
+        z = orc.router_logits(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]))
+        zt = torch.from_numpy(z).cuda()
+        for policy in (orc.SUBSTITUTION, orc.TRUNCATION):
+            for mode in (orc.FROM_ALL, orc.FROM_UNION):
+                for renorm in (True, False):
+                    layer = make_layer(case, max_M=M, max_k=cfg.k, policy=policy, shortlist=mode,
+                                       renormalize=renorm, ffn_kernel=ms().FFN_CUDA_CORE)
+                    for B in Bs:
+                        r = H.oracle_route(z, cfg.k, B, policy, mode, renorm)
+                        # certify the answer is unique at the GPU's fp64 scoring accuracy
+                        cand = None if mode == orc.FROM_ALL else r["union"]
+                        zgap, sgap = H.selection_margins(r, cfg.k, cand)
+                        assert sgap > 1e-10, "fixture has a score near-tie at the cut"
+                        layer.route_from_logits(zt, cfg.k, B)
+                        H.compare_routing(layer.get_routing(), r, policy, cfg.k)
+                        st = layer.get_stats()
+                        assert st["n_union"] == len(r["union"]) and st["n_active"] == len(r["active"])
+                        if mode == orc.FROM_UNION:
+                            assert st["n_shortlist"] == min(B, len(r["union"]))
+                        else:
+                            assert st["n_shortlist"] == min(B, cfg.n_experts)
+                    layer.destroy()
+
+
+def test_constructed_ties_resolve_to_lower_index():
+    cfg = synth.CONFIGS["tiny"]
+    case = H.make_case(cfg, 15, seed=2)
+    z = orc.router_logits(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]))
+    z[:, 9] = z[:, 3]          # identical columns: identical logits, probabilities and scores
+    z[:, 12] = z[:, 5]
+    z[4, :] = 0.25             # one token with all logits equal
+    zt = torch.from_numpy(z).cuda()
+    for policy in (orc.SUBSTITUTION, orc.TRUNCATION):
+        for mode in (orc.FROM_ALL, orc.FROM_UNION):
+            layer = make_layer(case, max_M=15, max_k=4, policy=policy, shortlist=mode, ffn_kernel=ms().FFN_CUDA_CORE)
+            for B in range(1, 17):
+                r = H.oracle_route(z, 4, B, policy, mode, True)
+                layer.route_from_logits(zt, 4, B)
+                H.compare_routing(layer.get_routing(), r, policy, 4)
+            layer.destroy()
+
+
+# ------------------------------------------------------------------ whole layer
+@pytest.mark.parametrize("policy", [orc.SUBSTITUTION, orc.TRUNCATION])
+@pytest.mark.parametrize("renorm", [True, False])
+def test_tiny_fp32_layer(policy, renorm):
+    cfg = synth.CONFIGS["tiny"]
+    for mode in (orc.FROM_ALL, orc.FROM_UNION):
+        for B in (2, 8, 16):
+            run_e2e(cfg, 15, B, policy, mode, renorm, ms().FFN_AUTO)
+
+
+@pytest.mark.parametrize("ffn", ["cuda_core", "tensor_core"])
+@pytest.mark.parametrize("B", [16, 32, 48, 64])
+def test_olmoe_layer_bf16(ffn, B):
+    cfg = synth.CONFIGS["olmoe"]
+    kern = ms().FFN_CUDA_CORE if ffn == "cuda_core" else ms().FFN_TENSOR_CORE
+    out, r, st = run_e2e(cfg, 63, B, orc.SUBSTITUTION, orc.FROM_ALL, True, kern)
+    assert st["n_rows"] == 63 * 8
+
+
+@pytest.mark.parametrize("M", [1, 7, 31, 77, 127, 255])
+def test_olmoe_tree_sizes_tensor_core(M):
+    cfg = synth.CONFIGS["olmoe"]
+    case = H.make_case(cfg, M, seed=M)
+    for B, policy in ((32, orc.SUBSTITUTION), (64, orc.SUBSTITUTION), (12, orc.TRUNCATION)):
+        run_e2e(cfg, M, B, policy, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, case=case)
+
+
+def test_token_chunking_beyond_256_rows_per_expert():
+    cfg = synth.CONFIGS["olmoe"].with_(n_experts=16, f=256, d=512)
+    # B = k: every token is routed to the same 8 experts, 300 rows each -> two token chunks per expert
+    out, r, st = run_e2e(cfg, 300, 8, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    assert max(r["count"]) == 300
+
+
+def test_qwen3_shape_layer():
+    cfg = synth.CONFIGS["qwen3"]
+    for M, B in ((63, 32), (127, 128)):
+        run_e2e(cfg, M, B, orc.SUBSTITUTION, orc.FROM_ALL, False, ms().FFN_TENSOR_CORE)
+
+
+def test_mixtral_shape_layer_reduced_width():
+    # full d and k/N of the Mixtral-shaped layer, FFN width reduced so the oracle finishes in seconds
+    cfg = synth.CONFIGS["mixtral"].with_(f=1792)
+    for M, B in ((15, 4), (63, 6)):
+        run_e2e(cfg, M, B, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+
+
+def test_truncation_zero_rows_and_budget_below_k():
+    cfg = synth.CONFIGS["olmoe"].with_(f=128, slope=0.0)      # flat routing: no expert is in every top-k
+    out, r, st = run_e2e(cfg, 63, 1, orc.TRUNCATION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    empty = [t for t in range(63) if not r["assign"][t]]
+    assert empty, "fixture should drop every expert of some token"
+    assert not out[empty].float().abs().max().item() > 0      # exact zeros
+    assert st["n_dropped"] > 0
+    out, r, st = run_e2e(cfg, 63, 3, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    assert st["n_rows"] == 63 * 3                              # B < k: min(k, |S|) experts per token
+
+
+def test_unbudgeted_identities_on_gpu():
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = H.make_case(cfg, 31, seed=4)
+    m = ms()
+    full = make_layer(case, 31, 8, policy=m.SUBSTITUTION, shortlist=m.FROM_ALL)
+    o_full = full.verify_layer(case["hidden"], 8, 64).clone()
+    o_over = full.verify_layer(case["hidden"], 8, 1000).clone()      # B > N clamps to N
+    assert torch.equal(o_full, o_over)
+    nE = full.get_stats()["n_union"]
+    uni = make_layer(case, 31, 8, policy=m.TRUNCATION, shortlist=m.FROM_UNION)
+    o_uni = uni.verify_layer(case["hidden"], 8, nE).clone()          # B = |E| under the union reading
+    assert uni.get_stats()["n_shortlist"] == nE
+    assert torch.equal(o_full, o_uni)
+    one = make_layer(case, 31, 8, policy=m.SUBSTITUTION, shortlist=m.FROM_ALL)
+    o1 = one.verify_layer(case["hidden"][:1].contiguous(), 8, 8).clone()   # M = 1, B = k
+    o1_full = one.verify_layer(case["hidden"][:1].contiguous(), 8, 64).clone()
+    assert torch.equal(o1, o1_full)
+    for L in (full, uni, one):
+        L.destroy()
+
+
+def test_residual_and_host_entry_point():
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = H.make_case(cfg, 63, seed=6)
+    run_e2e(cfg, 63, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, case=case, residual=True)
+    run_e2e(cfg, 63, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, case=case, residual=True,
+            out_dtype=torch.bfloat16)
+    run_e2e(cfg, 63, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, case=case, out_dtype=torch.bfloat16)
+    layer = make_layer(case, 63, 8)
+    dev = layer.verify_layer(case["hidden"], 8, 32).cpu()
+    h_host = case["hidden"].cpu().pin_memory()
+    o_host = torch.empty_like(h_host).pin_memory()
+    layer.verify_layer_host(h_host, 8, 32, o_host)
+    assert torch.equal(dev, o_host)
+    assert layer.last_launch_count() >= 5
+    layer.destroy()
+
+
+def test_repeat_calls_are_bitwise_reproducible():
+    cfg = synth.CONFIGS["olmoe"].with_(f=256)
+    case = H.make_case(cfg, 127, seed=8)
+    layer = make_layer(case, 127, 8)
+    a = layer.verify_layer(case["hidden"], 8, 32).clone()
+    layer.verify_layer(case["hidden"][:40].contiguous(), 8, 16)
+    b = layer.verify_layer(case["hidden"], 8, 32).clone()
+    assert torch.equal(a, b)
+    layer.destroy()
+
+
+# ------------------------------------------------------------------ argument errors (host side only)
+def test_argument_errors_return_codes():
+    m = ms()
+    cfg = synth.CONFIGS["tiny"]
+    case = H.make_case(cfg, 15)
+    layer = make_layer(case, max_M=15, max_k=4)
+    h, out = case["hidden"], torch.empty_like(case["hidden"])
+    lib, hd = m.lib(), layer._h
+    s = torch.cuda.current_stream().cuda_stream
+    assert lib.moespec_verify_layer(hd, h.data_ptr(), 16, 4, 8, out.data_ptr(), s) == m.ERR_INVALID_ARG   # M > max_M
+    assert lib.moespec_verify_layer(hd, h.data_ptr(), 15, 5, 8, out.data_ptr(), s) == m.ERR_INVALID_ARG   # k > max_k
+    assert lib.moespec_verify_layer(hd, h.data_ptr(), 15, 0, 8, out.data_ptr(), s) == m.ERR_INVALID_ARG
+    assert lib.moespec_verify_layer(hd, h.data_ptr(), 15, 4, 0, out.data_ptr(), s) == m.ERR_INVALID_ARG   # B < 1
+    assert lib.moespec_verify_layer(hd, None, 15, 4, 8, out.data_ptr(), s) == m.ERR_NULL_POINTER
+    assert lib.moespec_verify_layer(hd, h.data_ptr(), 15, 4, 8, h.data_ptr(), s) == m.ERR_INVALID_ARG     # aliasing
+    assert lib.moespec_verify_layer(hd, h.data_ptr() + 4, 14, 4, 8, out.data_ptr(), s) == m.ERR_UNSUPPORTED
+    assert lib.moespec_verify_layer(hd, None, 0, 4, 8, None, s) == m.OK                                   # M = 0 no-op
+    assert lib.moespec_verify_layer(None, h.data_ptr(), 15, 4, 8, out.data_ptr(), s) == m.ERR_BAD_HANDLE
+    raw = hd.value
+    layer.destroy()
+    assert lib.moespec_verify_layer(raw, h.data_ptr(), 15, 4, 8, out.data_ptr(), s) == m.ERR_BAD_HANDLE   # destroyed
+    assert lib.moespec_destroy(raw) == m.ERR_BAD_HANDLE
+    with pytest.raises(m.MoeSpecError):
+        make_layer(case, max_M=15, max_k=4, policy=0)
+    with pytest.raises(m.MoeSpecError):
+        make_layer(case, max_M=15, max_k=4, shortlist=0)
+    with pytest.raises(m.MoeSpecError):
+        make_layer(case, max_M=15, max_k=4, ffn_kernel=m.FFN_TENSOR_CORE)    # fp32 has no tensor-core kernel
+    torch.cuda.synchronize()
