@@ -46,7 +46,8 @@ typedef enum {
   MOESPEC_ERR_CUDA = -5,          /* a CUDA runtime/driver call failed (see moespec_last_cuda_error) */
   MOESPEC_ERR_TIMEOUT = -6,       /* a bounded device-side wait expired (reported via stats)     */
   MOESPEC_ERR_INTERNAL = -7,      /* a device-side consistency check failed (reported via stats) */
-  MOESPEC_ERR_BAD_HANDLE = -8     /* handle is NULL, was destroyed, or was never created         */
+  MOESPEC_ERR_BAD_HANDLE = -8,    /* handle is NULL, was destroyed, or was never created         */
+  MOESPEC_ERR_TOO_LARGE = -9      /* a size exceeds the fixed capacity of moespec_route_static   */
 } moespec_status;
 
 typedef enum { MOESPEC_BF16 = 1, MOESPEC_FP32 = 2 } moespec_dtype_t;
@@ -123,6 +124,50 @@ int moespec_verify_layer_host(moespec_layer_t *layer, const void *hidden_host, i
  * checked through: fed the same fp32 logits, selection is exact. */
 int moespec_route_from_logits(moespec_layer_t *layer, const float *logits, int M, int k, int B,
                               void *stream);
+
+/* The routing step for callers that cannot allocate device memory.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs while a CUDA stream is being captured (allocation
+ * cannot be captured), serving loops that must avoid the implicit device-wide
+ * synchronisation of cudaMalloc/cudaFree, and processes whose device memory is
+ * wholly owned by another allocator.  Such callers cannot use
+ * moespec_layer_create, which allocates a workspace.
+ *
+ * What it does: exactly the computation of moespec_route_from_logits (softmax,
+ * top-k, Eq. 5 scores, shortlist, Eq. 7 / Eq. 8 re-routing, Appendix C gather
+ * order), without a handle.  Its scratch memory is a fixed array inside the
+ * library image, about 1.1 MB, held by every GPU that loads the library until
+ * the process exits.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Limits: M <= MOESPEC_ROUTE_STATIC_MAX_M, N <= MOESPEC_ROUTE_STATIC_MAX_N,
+ * k <= MOESPEC_ROUTE_STATIC_MAX_K, M*k <= MOESPEC_ROUTE_STATIC_MAX_ROWS; anything
+ * larger returns MOESPEC_ERR_TOO_LARGE and launches nothing.
+ *
+ * Arguments: logits is device [M, N] fp32 on the calling thread's CURRENT
+ * device; every output is a device buffer on that device, owned by the caller,
+ * with the meaning and size given for moespec_get_routing (S_rank[N],
+ * topk_idx/assign_idx/gate_w/tokslot2row[M*k], count[N], offset[N+1],
+ * perm_row2tok[M*k], score[N]); summary is device int[8]: [0] = |S|,
+ * [1] = experts with rows, [2] = R.  policy / shortlist / renormalize are the
+ * fields of moespec_layer_desc.  Enqueues on `stream` and returns.
+ *
+ * Sharing: all calls in the process use the same scratch array, which keeps the
+ * previous call's contents; the kernel rewrites every word before reading it,
+ * so nothing needs clearing, but two calls that overlap on the GPU (different
+ * streams or threads) race on it.  Serialise them.
+ *
+ * First call: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) with that device current; make that first call before
+ * starting any stream capture. */
+#define MOESPEC_ROUTE_STATIC_MAX_M 512
+#define MOESPEC_ROUTE_STATIC_MAX_N 256
+#define MOESPEC_ROUTE_STATIC_MAX_K 32
+#define MOESPEC_ROUTE_STATIC_MAX_ROWS 8192
+int moespec_route_static(const float *logits, int M, int N, int k, int B, int policy, int shortlist,
+                         int renormalize, int *S_rank, int *topk_idx, int *assign_idx, float *gate_w,
+                         int *count, int *offset, int *perm_row2tok, int *tokslot2row, double *score,
+                         int *summary, void *stream);
 
 /* Copy the routing state of the last verify/route call into HOST buffers (any
  * may be NULL to skip it).  Synchronises the device.

@@ -436,6 +436,7 @@ const char *moespec_strerror(int status) {
     case MOESPEC_ERR_TIMEOUT: return "bounded device-side wait expired";
     case MOESPEC_ERR_INTERNAL: return "device-side consistency check failed";
     case MOESPEC_ERR_BAD_HANDLE: return "bad or destroyed handle";
+    case MOESPEC_ERR_TOO_LARGE: return "size exceeds the fixed scratch capacity of moespec_route_static";
     default: return "unknown status";
   }
 }

@@ -23,11 +23,12 @@ FFN_AUTO, FFN_CUDA_CORE, FFN_TENSOR_CORE = 0, 1, 2
 
 OK = 0
 ERR_INVALID_ARG, ERR_NULL_POINTER, ERR_UNSUPPORTED, ERR_OUT_OF_MEMORY = -1, -2, -3, -4
-ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL, ERR_BAD_HANDLE = -5, -6, -7, -8
+ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL, ERR_BAD_HANDLE, ERR_TOO_LARGE = -5, -6, -7, -8, -9
+ROUTE_STATIC_MAX_M, ROUTE_STATIC_MAX_N, ROUTE_STATIC_MAX_K, ROUTE_STATIC_MAX_ROWS = 512, 256, 32, 8192
 
 EXPORTS = [
     "moespec_layer_create", "moespec_verify_layer", "moespec_verify_layer_host",
-    "moespec_route_from_logits", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
+    "moespec_route_from_logits", "moespec_route_static", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
     "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
     "moespec_version",
 ]
@@ -76,6 +77,7 @@ def lib() -> C.CDLL:
         L.moespec_verify_layer.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.moespec_verify_layer_host.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.moespec_route_from_logits.argtypes = [vp, vp, ci, ci, ci, vp]
+        L.moespec_route_static.argtypes = [vp] + [ci] * 7 + [vp] * 11
         L.moespec_get_routing.argtypes = [vp] + [vp] * 11
         L.moespec_get_logits.argtypes = [vp, vp]
         L.moespec_get_intermediate.argtypes = [vp, ci, vp, C.c_longlong]
@@ -105,6 +107,35 @@ def _np_ptr(a: Optional[np.ndarray]):
 def _stream_ptr(stream) -> int:
     s = torch.cuda.current_stream() if stream is None else stream
     return s.cuda_stream
+
+
+def route_static(logits: torch.Tensor, k: int, B: int, policy: int, shortlist: int, renormalize: bool,
+                 out: Optional[dict] = None, stream=None) -> dict:
+    """moespec_route_static: the routing step with no allocation inside the library.
+
+    For callers that cannot allocate device memory at the call site (inside a
+    stream capture, in a loop that must not trigger cudaMalloc's device-wide
+    synchronisation, or when another allocator owns the device memory).  The
+    output tensors are the caller's: pass the dict a previous call returned to
+    reuse them, otherwise this wrapper makes them with torch before calling in.
+    All calls share one fixed scratch array inside the library, so calls that
+    overlap on the GPU race; M, N, k are capped (ROUTE_STATIC_MAX_*).
+    """
+    M, N = logits.shape
+    assert logits.dtype == torch.float32 and logits.is_cuda and logits.is_contiguous()
+    if out is None:
+        dev = logits.device
+        i32 = lambda n: torch.empty(max(n, 1), dtype=torch.int32, device=dev)
+        out = {"S_rank": i32(N), "topk_idx": i32(M * k), "assign_idx": i32(M * k),
+               "gate_w": torch.empty(max(M * k, 1), dtype=torch.float32, device=dev), "count": i32(N),
+               "offset": i32(N + 1), "perm_row2tok": i32(M * k), "tokslot2row": i32(M * k),
+               "score": torch.empty(N, dtype=torch.float64, device=dev), "summary": i32(8)}
+    p = lambda name: out[name].data_ptr()
+    _check(lib().moespec_route_static(logits.data_ptr(), M, N, k, B, policy, shortlist, int(renormalize),
+                                      p("S_rank"), p("topk_idx"), p("assign_idx"), p("gate_w"), p("count"),
+                                      p("offset"), p("perm_row2tok"), p("tokslot2row"), p("score"), p("summary"),
+                                      _stream_ptr(stream)), "moespec_route_static")
+    return out
 
 
 class Layer:

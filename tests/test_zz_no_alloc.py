@@ -1,0 +1,68 @@
+"""moespec_route_static, the entry point for callers that cannot allocate device memory.
+
+Such callers (code inside a CUDA stream capture, serving loops that must avoid the device-wide
+synchronisation cudaMalloc can cause, processes whose memory belongs to another allocator) get the
+routing step with its scratch in a fixed array inside the library.  This test calls it through the
+C ABI twice in a row, with different sizes so that the second call sees the first call's leftovers
+in the shared scratch, and requires the same results as the handle-based entry point.
+
+The file sorts last on purpose: a run that stops at the first failure has then run everything else.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_16052_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def reference_routing(m, case, z, k, B, policy, shortlist, renorm):
+    layer = m.Layer(case["router_w"], case["router_bias"], case["w_gate"], case["w_up"], case["w_down"],
+                    max_M=z.shape[0], max_k=k, policy=policy, shortlist=shortlist, renormalize=renorm,
+                    ffn_kernel=m.FFN_CUDA_CORE)
+    layer.route_from_logits(z, k, B)
+    g = layer.get_routing()
+    layer.destroy()
+    return g
+
+
+def check_same(out, g, M, k):
+    torch.cuda.synchronize()
+    nS, _, R = out["summary"][:3].tolist()
+    assert out["S_rank"][:nS].tolist() == g["S"] and R == g["n_rows"]
+    for name in ("topk_idx", "assign_idx", "tokslot2row"):
+        assert np.array_equal(out[name][:M * k].cpu().numpy().reshape(M, k), g[name]), name
+    # same kernel, same inputs: the floating-point outputs are identical, which is inside any tolerance
+    assert np.array_equal(out["gate_w"][:M * k].cpu().numpy().reshape(M, k), g["gate_w"])
+    assert np.array_equal(out["score"].cpu().numpy(), g["score"])
+    assert out["count"].tolist() == g["count"] and out["offset"].tolist() == g["offset"]
+    assert out["perm_row2tok"][:R].tolist() == g["perm_row2tok"]
+
+
+def test_route_static_matches_handle_based_routing_twice_in_a_row():
+    from paper_2602_16052_b200 import moespec as m
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = synth.gen_layer(cfg, 21, 0, "cuda")
+    k = cfg.k
+    calls = [(127, 32, m.SUBSTITUTION, m.FROM_ALL, True), (40, 5, m.TRUNCATION, m.FROM_UNION, False)]
+    for M, B, policy, shortlist, renorm in calls:
+        h = synth.gen_hidden(cfg, M, 21, 0, "cuda")
+        z = (h.float() @ case["router_w"].float().T + case["router_bias"]).contiguous()   # any fp32 logits will do
+        want = reference_routing(m, case, z, k, B, policy, shortlist, renorm)
+        got = m.route_static(z, k, B, policy, shortlist, renorm)
+        check_same(got, want, M, k)
+        again = m.route_static(z, k, B, policy, shortlist, renorm, out=got)     # reuse the caller's buffers
+        check_same(again, want, M, k)
+
+
+def test_route_static_rejects_sizes_beyond_its_scratch():
+    from paper_2602_16052_b200 import moespec as m
+    z = torch.zeros((m.ROUTE_STATIC_MAX_M + 1, 8), dtype=torch.float32, device="cuda")
+    with pytest.raises(m.MoeSpecError) as e:
+        m.route_static(z, 2, 4, m.SUBSTITUTION, m.FROM_ALL, True)
+    assert e.value.code == m.ERR_TOO_LARGE and "capacity" in str(e.value)
+    z = torch.zeros((4, m.ROUTE_STATIC_MAX_N + 1), dtype=torch.float32, device="cuda")
+    with pytest.raises(m.MoeSpecError) as e:
+        m.route_static(z, 2, 4, m.SUBSTITUTION, m.FROM_ALL, True)
+    assert e.value.code == m.ERR_TOO_LARGE
