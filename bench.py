@@ -248,6 +248,9 @@ def main():
     ap.add_argument("--impl", default="moespec", choices=["moespec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--copies", type=int, default=N_COPIES, help="independently seeded layer copies rotated over")
+    ap.add_argument("--timed-only", action="store_true",
+                    help="run only the warm-up and the timed steps (for profiler captures); prints a short line")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -281,7 +284,7 @@ def main():
     cfg = synth.CONFIGS[WORKLOAD]
     M, k, B = M_TOKENS, cfg.k, B_HEADLINE
     out_dtype = torch.float32          # unrounded fp32 accumulators, the output the 2e-2*RMS bar is stated on
-    layers, hiddens = build_layers(cfg, M, N_COPIES, device, out_dtype)
+    layers, hiddens = build_layers(cfg, M, args.copies, device, out_dtype)
     outs = [torch.empty((M, cfg.d), dtype=out_dtype, device=device) for _ in layers]
 
     sampler = ClockSampler(local_rank)
@@ -295,6 +298,13 @@ def main():
     launches_per_step = layers[0].last_launch_count()
     stats = layers[0].get_stats()
     assert stats["status"] == 0, stats
+
+    if args.timed_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": ms_total * 1e3 / (args.steps * world), "unit": "us",
+                              "steps": args.steps, "warmup": args.warmup, "timed_only": True,
+                              "gpu_launches": launches_per_step * args.steps}), flush=True)
+        return
 
     e2e_ms, h2d, d2h = time_e2e(layers, hiddens, k, B, args.steps, args.warmup, out_dtype)
     e2e_ms = max_over_ranks(e2e_ms)
@@ -346,8 +356,8 @@ def main():
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": False,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(cfg),
-                       "l2": f"rotating over {N_COPIES} independently seeded layer copies "
-                             f"({N_COPIES * cfg.n_experts * cfg.expert_weight_bytes() / 1e9:.1f} GB); each step streams "
+                       "l2": f"rotating over {args.copies} independently seeded layer copies "
+                             f"({args.copies * cfg.n_experts * cfg.expert_weight_bytes() / 1e9:.1f} GB); each step streams "
                              f"{ffn_bytes / 1e6:.0f} MB > 126 MB L2",
                        "replicas": world, "n_active": mean_active, "n_union": stats["n_union"],
                        "coverage": stats["coverage"]},

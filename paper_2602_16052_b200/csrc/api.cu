@@ -1,6 +1,7 @@
 // C ABI of libmoespec: handle life cycle, argument validation, workspace, launch order.
 #include "internal.h"
 
+#include <cstdlib>
 #include <mutex>
 #include <new>
 #include <unordered_set>
@@ -101,6 +102,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.tokslot2row, M * K);
   c.take(w.natmask, M * kMaskWords);
   c.take(w.amask, M * kMaskWords);
+  c.take(w.arrive, M);
   c.take(w.units_up, max_chunks * tiles_up);
   c.take(w.units_down, max_chunks * tiles_down);
   c.take(w.counters, 16);
@@ -127,7 +129,7 @@ bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream};
-  int launches = 0, n = 0;
+  int launches = 0;
   cudaError_t e;
   // with profiling on, an event is recorded before the first kernel and after every kernel
   auto mark = [&](int i) -> cudaError_t {
@@ -136,7 +138,7 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   if ((e = mark(0)) != cudaSuccess) return cuda_fail(e);
   if ((e = launch_router_logits(c, hidden)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
-  if ((e = launch_route(c, L->ws.logits)) != cudaSuccess) return cuda_fail(e);
+  if ((e = launch_route_after_router(c)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
@@ -153,7 +155,6 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   }
   if ((e = launch_combine(c, hidden, out)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
-  (void)n;
   L->last_M = M;
   L->last_k = k;
   L->last_launches = launches;
@@ -161,6 +162,16 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
 }
 
 }  // namespace
+
+namespace moespec {
+bool pdl_enabled() {
+  static const bool on = [] {
+    const char *v = getenv("MOESPEC_NO_PDL");
+    return !(v && v[0] == '1');
+  }();
+  return on;
+}
+}  // namespace moespec
 
 extern "C" {
 
@@ -296,7 +307,7 @@ int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, in
   if (e != cudaSuccess) return cuda_fail(e);
   L->last_M = M;
   L->last_k = k;
-  L->last_launches = 1;
+  L->last_launches = 2;
   return MOESPEC_OK;
 }
 

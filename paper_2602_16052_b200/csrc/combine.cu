@@ -32,6 +32,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
   const int t = blockIdx.x;
   __shared__ int s_row[kMaxK];
   __shared__ float s_w[kMaxK];
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x < k) {
     s_row[threadIdx.x] = tokslot2row[(size_t)t * k + threadIdx.x];
     s_w[threadIdx.x] = gate_w[(size_t)t * k + threadIdx.x];
@@ -58,19 +60,19 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
 }
 
 template <typename T, typename TO>
-static void launch_t(const LaunchCtx &c, const void *hidden, void *out) {
+static cudaError_t launch_t(const LaunchCtx &c, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
-  combine_kernel<T, TO><<<c.M, 256, 0, c.stream>>>(c.ws->y, c.ws->gate_w, c.ws->tokslot2row, (const T *)hidden,
-                                                   (TO *)out, D.d, c.k, D.residual);
+  return launch_kernel(combine_kernel<T, TO>, dim3(c.M), dim3(256), 0, c.stream, (const float *)c.ws->y,
+                       (const float *)c.ws->gate_w, (const int *)c.ws->tokslot2row, (const T *)hidden, (TO *)out, D.d,
+                       c.k, D.residual);
 }
 
 cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
   const int od = D.out_dtype ? D.out_dtype : D.dtype;
-  if (D.dtype == MOESPEC_BF16 && od == MOESPEC_BF16) launch_t<__nv_bfloat16, __nv_bfloat16>(c, hidden, out);
-  else if (D.dtype == MOESPEC_BF16) launch_t<__nv_bfloat16, float>(c, hidden, out);
-  else launch_t<float, float>(c, hidden, out);
-  return cudaGetLastError();
+  if (D.dtype == MOESPEC_BF16 && od == MOESPEC_BF16) return launch_t<__nv_bfloat16, __nv_bfloat16>(c, hidden, out);
+  if (D.dtype == MOESPEC_BF16) return launch_t<__nv_bfloat16, float>(c, hidden, out);
+  return launch_t<float, float>(c, hidden, out);
 }
 
 }  // namespace moespec

@@ -22,6 +22,8 @@ __global__ void __launch_bounds__(256) ffn_gateup_cc_kernel(const T *__restrict_
                                                             const int *__restrict__ counters, int d, int f) {
   extern __shared__ float xs[];
   const int r = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   if (r >= counters[2]) return;
   const int e = row2expert[r];
   const T *x = x_perm + (size_t)r * d;
@@ -63,6 +65,8 @@ __global__ void __launch_bounds__(256) ffn_down_cc_kernel(const T *__restrict__ 
                                                           const int *__restrict__ counters, int d, int f) {
   extern __shared__ float ms[];
   const int r = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   if (r >= counters[2]) return;
   const int e = row2expert[r];
   const T *m = h_mid + (size_t)r * f;
@@ -93,15 +97,15 @@ static cudaError_t launch_cc(const LaunchCtx &c, int phase) {
   const int rows = c.M * c.k;
   if (phase == 0) {
     dim3 g1(rows, (D.f + kColsPerBlock - 1) / kColsPerBlock);
-    ffn_gateup_cc_kernel<T><<<g1, 256, D.d * sizeof(float), c.stream>>>(
-        (const T *)c.ws->x_perm, (const T *)D.w_gate, (const T *)D.w_up, (T *)c.ws->h_mid, c.ws->row2expert,
-        c.ws->counters, D.d, D.f);
+    return launch_kernel(ffn_gateup_cc_kernel<T>, g1, dim3(256), D.d * sizeof(float), c.stream,
+                         (const T *)c.ws->x_perm, (const T *)D.w_gate, (const T *)D.w_up, (T *)c.ws->h_mid,
+                         (const int *)c.ws->row2expert, (const int *)c.ws->counters, D.d, D.f);
   } else {
     dim3 g2(rows, (D.d + kColsPerBlock - 1) / kColsPerBlock);
-    ffn_down_cc_kernel<T><<<g2, 256, D.f * sizeof(float), c.stream>>>(
-        (const T *)c.ws->h_mid, (const T *)D.w_down, c.ws->y, c.ws->row2expert, c.ws->counters, D.d, D.f);
+    return launch_kernel(ffn_down_cc_kernel<T>, g2, dim3(256), D.f * sizeof(float), c.stream,
+                         (const T *)c.ws->h_mid, (const T *)D.w_down, c.ws->y, (const int *)c.ws->row2expert,
+                         (const int *)c.ws->counters, D.d, D.f);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase) {

@@ -42,7 +42,8 @@ struct TcArgs {
   const Unit *units;
   const int *n_units;
   int phase;            // 0 gate/up, 1 down
-  int k_chunks;         // K / 64
+  int k_iters;          // ring stages per unit: K/64 in phase 0 (gate chunk + up chunk), K/128 in phase 1
+  int b1_off;           // phase 1: offset of the second token slab inside a stage
   int n_stages;
   int stage_bytes;
   int acc_bufs;         // 1 or 2 accumulator buffers of 256 TMEM columns
@@ -162,8 +163,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + 16 * kMaxStages + 36);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_units = *a.n_units;
   const int n_stages = a.n_stages;
+  pdl_trigger();
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -188,11 +189,15 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above overlaps the tail of the previous kernel; its results are read from here on
+  pdl_wait();
+  const int n_units = *a.n_units;
 
   const CUtensorMap *map_a0 = a.phase == 0 ? &maps.w_gate : &maps.w_down;
   const CUtensorMap *map_a1 = &maps.w_up;
   const CUtensorMap *map_b = a.phase == 0 ? &maps.x_perm : &maps.h_mid;
-  const uint32_t a_bytes = a.phase == 0 ? 2u * kABytes : (uint32_t)kABytes;
+  // every stage carries 32 KB of weights: phase 0 one K chunk of gate and of up, phase 1 two K chunks of down
+  const uint32_t b_slabs = a.phase == 0 ? 1u : 2u;
 
   if (warp == 0 && lane == 0) {
     // ===================================================== TMA producer
@@ -201,16 +206,26 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
       const Unit un = a.units[u];
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
-      for (int kc = 0; kc < a.k_chunks; ++kc, ++it) {
+      for (int kc = 0; kc < a.k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t full = bar_full + 8 * s;
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
-        mbar_expect_tx(full, a_bytes + (uint32_t)n_pad * 128u);
-        tma_load_3d(stage, map_a0, full, kc * kChunkK, un.tile * kTile, un.expert);
-        if (a.phase == 0) tma_load_3d(stage + kABytes, map_a1, full, kc * kChunkK, un.tile * kTile, un.expert);
-        for (int b = 0; b < n_pad / kTokBox; ++b)
-          tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
+        mbar_expect_tx(full, 2u * kABytes + b_slabs * (uint32_t)n_pad * 128u);
+        if (a.phase == 0) {
+          tma_load_3d(stage, map_a0, full, kc * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage + kABytes, map_a1, full, kc * kChunkK, un.tile * kTile, un.expert);
+          for (int b = 0; b < n_pad / kTokBox; ++b)
+            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
+        } else {
+          tma_load_3d(stage, map_a0, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage + kABytes, map_a0, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert);
+          for (int b = 0; b < n_pad / kTokBox; ++b) {
+            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, (2 * kc) * kChunkK, un.row0 + b * kTokBox);
+            tma_load_2d(stage + a.b1_off + b * (kTokBox * 128), map_b, full, (2 * kc + 1) * kChunkK,
+                        un.row0 + b * kTokBox);
+          }
+        }
       }
     }
     if (!ok) {
@@ -234,18 +249,29 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const uint32_t tmem_d = tmem_base + ab * 256u;
-      for (int kc = 0; kc < a.k_chunks; ++kc, ++it) {
+      for (int kc = 0; kc < a.k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
+        if (a.phase == 0) {
 #pragma unroll
-        for (int kk = 0; kk < kChunkK / 16; ++kk) {
-          const uint32_t acc = (kc > 0 || kk > 0) ? 1u : 0u;
-          const uint64_t bdesc = smem_desc_sw128(stage + kBOffset + kk * 32);
-          tc_mma_bf16(tmem_d, smem_desc_sw128(stage + kk * 32), bdesc, idesc, acc);
-          if (a.phase == 0)
+          for (int kk = 0; kk < kChunkK / 16; ++kk) {
+            const uint32_t acc = (kc > 0 || kk > 0) ? 1u : 0u;
+            const uint64_t bdesc = smem_desc_sw128(stage + kBOffset + kk * 32);
+            tc_mma_bf16(tmem_d, smem_desc_sw128(stage + kk * 32), bdesc, idesc, acc);
             tc_mma_bf16(tmem_d + (uint32_t)n_pad, smem_desc_sw128(stage + kABytes + kk * 32), bdesc, idesc, acc);
+          }
+        } else {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+            const uint32_t a_off = stage + half * kABytes;
+            const uint32_t b_off = stage + (half ? (uint32_t)a.b1_off : (uint32_t)kBOffset);
+#pragma unroll
+            for (int kk = 0; kk < kChunkK / 16; ++kk)
+              tc_mma_bf16(tmem_d, smem_desc_sw128(a_off + kk * 32), smem_desc_sw128(b_off + kk * 32), idesc,
+                          (kc > 0 || half > 0 || kk > 0) ? 1u : 0u);
+          }
         }
         tc_commit(bar_empty + 8 * s);      // stage reusable once these MMAs have read it
       }
@@ -367,29 +393,29 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, int p
   const moespec_layer_desc &D = *c.desc;
   const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
   TcArgs a;
-  a.stage_bytes = kBOffset + n_pad_max * 128;
+  a.phase = phase;
+  a.b1_off = kBOffset + n_pad_max * 128;
+  a.stage_bytes = kBOffset + (phase == 0 ? 1 : 2) * n_pad_max * 128;
   int stages = (kSmemBudget - 1024 - kCtrlBytes) / a.stage_bytes;
   a.n_stages = stages > kMaxStages ? kMaxStages : stages;
   a.acc_bufs = 2 * n_pad_max <= 256 ? 2 : 1;
   a.status = c.ws->status;
   const int grid = sm_count_cached(D.device);
   const size_t smem = (size_t)a.n_stages * a.stage_bytes + 1024 + kCtrlBytes;
-  a.phase = phase;
   if (phase == 0) {
     a.units = c.ws->units_up;
     a.n_units = c.ws->counters + 3;
-    a.k_chunks = D.d / kChunkK;
+    a.k_iters = D.d / kChunkK;
     a.out = c.ws->h_mid;
     a.out_ld = D.f;
   } else {
     a.units = c.ws->units_down;
     a.n_units = c.ws->counters + 4;
-    a.k_chunks = D.f / kChunkK;
+    a.k_iters = D.f / (2 * kChunkK);
     a.out = c.ws->y;
     a.out_ld = D.d;
   }
-  ffn_tc_kernel<<<grid, kThreads, smem, c.stream>>>(*maps, a);
-  return cudaGetLastError();
+  return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, *maps, a);
 }
 
 }  // namespace moespec

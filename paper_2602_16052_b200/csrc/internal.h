@@ -41,6 +41,7 @@ struct Workspace {
   int *tokslot2row;     // [max_M, max_k]
   unsigned *natmask;    // [max_M, 8] bit i of row t: expert i in T_k(h_t)
   unsigned *amask;      // [max_M, 8] bit i of row t: expert i in A(t)
+  int *arrive;          // [max_M] per-token arrival counters of router_topk_kernel (zero between calls)
   Unit *units_up;       // gate/up units
   Unit *units_down;     // down units
   int *counters;        // [0]=n_S [1]=n_active [2]=R [3]=n_units_up [4]=n_units_down
@@ -61,9 +62,39 @@ struct LaunchCtx {
   cudaStream_t stream;
 };
 
+// Programmatic dependent launch.  Every kernel of the layer is launched with
+// programmatic stream serialisation: it may be scheduled while its predecessor
+// still runs, executes pdl_trigger() at once (so that its own successor can be
+// scheduled too) and calls pdl_wait() before it touches anything a predecessor
+// wrote or a predecessor may still read.  pdl_wait() returns when all earlier
+// kernels in the stream have completed and flushed; without the launch
+// attribute both calls are no-ops.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+bool pdl_enabled();   // false when MOESPEC_NO_PDL=1 is set in the environment
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                          Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // routing.cu
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden);
-cudaError_t launch_route(const LaunchCtx &c, const float *logits);
+cudaError_t launch_route(const LaunchCtx &c, const float *logits);   // softmax/top-k kernel + route kernel
+cudaError_t launch_route_after_router(const LaunchCtx &c);           // route kernel only
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
 // ffn_simple.cu
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down

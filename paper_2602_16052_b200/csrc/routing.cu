@@ -3,90 +3,201 @@
 // top-B shortlist (Section 3.2), re-routing under substitution (Eq. 8) or
 // truncation (Eq. 7) with the mixing weights of Section 3.3, and the
 // per-expert gather order (Appendix C).
+//
+// Two launches:
+//   router_topk_kernel   one warp per (token, expert) dot product; the CTA that
+//                        finishes a token's last logit also runs that token's
+//                        softmax and top-k (a counter, never a wait)
+//   route_kernel         one CTA: scores, shortlist, re-routing, scan, gather
+//                        order, work-unit list, statistics
+// A stand-alone softmax/top-k kernel serves callers that inject logits.
 #include "internal.h"
 #include <math_constants.h>
+#include <stdio.h>
 
 namespace moespec {
 
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
+constexpr unsigned kFull = 0xffffffffu;
+constexpr int kNone = 0x7fffffff;
+
+// Monotone map float -> uint32 (larger float, larger key); -0 and +0 share a key.
+__device__ __forceinline__ uint32_t order_key(float f) {
+  if (f == 0.f) f = 0.f;
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
 // ---------------------------------------------------------------------------
-// K1a: z[t,i] = b_i + w_i . h_t, fp32 accumulation.  One CTA per token; the
-// token row is staged in shared memory as fp32, each warp takes experts
-// warp, warp+8, ... and reads the router row with 16-byte loads.
+// Warp-wide ranking under (value descending, expert index ascending).  Lane l
+// owns experts l, l+32, ...; `valid` has bit s set while local slot s is still
+// a candidate.  Each round is two warp reductions: the maximum key, then the
+// lowest expert index among the lanes that hold it.  Winner r is returned in
+// lane r (-1 when fewer than r+1 candidates existed); winners leave `valid`.
+// ---------------------------------------------------------------------------
+template <int W>
+__device__ __forceinline__ int warp_take_best(const uint32_t (&key)[W], uint32_t &valid, int rounds, int lane) {
+  int mine = -1;
+  for (int r = 0; r < rounds; ++r) {
+    uint32_t bk = 0;
+    int bi = kNone;
+#pragma unroll
+    for (int s = 0; s < W; ++s)
+      if (((valid >> s) & 1u) && (bi == kNone || key[s] > bk)) { bk = key[s]; bi = lane + 32 * s; }
+    const uint32_t mk = __reduce_max_sync(kFull, bi == kNone ? 0u : bk);
+    const int win = __reduce_min_sync(kFull, (bi != kNone && bk == mk) ? bi : kNone);
+    if (win == kNone) break;
+    if ((win & 31) == lane) valid &= ~(1u << (win >> 5));
+    if (lane == r) mine = win;
+  }
+  return mine;
+}
+
+// Softmax (Eq. 1, fp64) and natural top-k (Eq. 2) of one token by one warp.
+template <int W>
+__device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int k, double *prob_row, int *topk_row,
+                                                   int lane) {
+  float v[W];
+  uint32_t key[W];
+  uint32_t valid = 0;
+  float mx = -CUDART_INF_F;
+#pragma unroll
+  for (int s = 0; s < W; ++s) {
+    const int idx = lane + 32 * s;
+    v[s] = -CUDART_INF_F;
+    key[s] = 0;
+    if (idx < N) {
+      v[s] = __ldcg(zrow + idx);          // written by other CTAs of this launch: read through L2
+      key[s] = order_key(v[s]);
+      valid |= 1u << s;
+      mx = fmaxf(mx, v[s]);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, o));
+  double e[W], sum = 0.0;
+#pragma unroll
+  for (int s = 0; s < W; ++s) {
+    e[s] = 0.0;
+    if ((valid >> s) & 1u) { e[s] = exp((double)v[s] - (double)mx); sum += e[s]; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
+#pragma unroll
+  for (int s = 0; s < W; ++s)
+    if ((valid >> s) & 1u) prob_row[lane + 32 * s] = e[s] / sum;
+  const int mine = warp_take_best<W>(key, valid, k, lane);
+  if (lane < k) topk_row[lane] = mine;
+}
+
+__device__ __forceinline__ void token_phase(const float *zrow, int N, int k, double *prob_row, int *topk_row, int lane) {
+  if (N <= 32) token_softmax_topk<1>(zrow, N, k, prob_row, topk_row, lane);
+  else if (N <= 64) token_softmax_topk<2>(zrow, N, k, prob_row, topk_row, lane);
+  else if (N <= 128) token_softmax_topk<4>(zrow, N, k, prob_row, topk_row, lane);
+  else token_softmax_topk<8>(zrow, N, k, prob_row, topk_row, lane);
+}
+
+// ---------------------------------------------------------------------------
+// K1: z[t,i] = b_i + w_i . h_t with fp32 accumulation, fused with the token's
+// softmax and top-k.  Grid (ceil(N/8), M): one warp per (token, expert) pair;
+// both rows are read with 16-byte loads issued before the first FMA.  Each CTA
+// then bumps the token's arrival counter; the CTA that sees the final count
+// finishes the token and resets the counter for the next call.
 // ---------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) router_logits_kernel(const T *__restrict__ hidden,
-                                                            const T *__restrict__ Wr,
-                                                            const float *__restrict__ bias,
-                                                            float *__restrict__ logits, int N, int d) {
-  extern __shared__ float xs[];
-  const int t = blockIdx.x;
-  const T *h = hidden + (size_t)t * d;
-  for (int j = threadIdx.x; j < d; j += blockDim.x) xs[j] = to_float(h[j]);
-  __syncthreads();
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  constexpr int VEC = 16 / sizeof(T);
-  for (int i = warp; i < N; i += nwarps) {
+__global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
+                                                          const float *__restrict__ bias, float *logits,
+                                                          double *prob, int *topk_idx, int *arrive, int N, int d,
+                                                          int k) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.y;
+  const int i = blockIdx.x * 8 + warp;
+  __shared__ int s_last;
+  pdl_trigger();
+  pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  if (i < N) {
+    constexpr int VEC = 16 / sizeof(T);
+    constexpr int U = 8;
+    const T *h = hidden + (size_t)t * d;
     const T *w = Wr + (size_t)i * d;
     float acc = 0.f;
-    for (int j = lane * VEC; j < d; j += 32 * VEC) {
-      uint4 raw = *reinterpret_cast<const uint4 *>(w + j);
-      const T *e = reinterpret_cast<const T *>(&raw);
+    for (int j0 = lane * VEC; j0 < d; j0 += 32 * VEC * U) {
+      uint4 rw[U], rh[U];
 #pragma unroll
-      for (int v = 0; v < VEC; ++v) acc = fmaf(to_float(e[v]), xs[j + v], acc);
+      for (int u = 0; u < U; ++u) {
+        const int j = j0 + u * 32 * VEC;
+        if (j < d) {
+          rw[u] = *reinterpret_cast<const uint4 *>(w + j);
+          rh[u] = *reinterpret_cast<const uint4 *>(h + j);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int j = j0 + u * 32 * VEC;
+        if (j < d) {
+          const T *ew = reinterpret_cast<const T *>(&rw[u]);
+          const T *eh = reinterpret_cast<const T *>(&rh[u]);
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) acc = fmaf(to_float(ew[v]), to_float(eh[v]), acc);
+        }
+      }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) logits[(size_t)t * N + i] = acc + (bias ? bias[i] : 0.f);
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
+    if (lane == 0) {
+      logits[(size_t)t * N + i] = acc + (bias ? bias[i] : 0.f);
+      __threadfence();
+    }
   }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(&arrive[t], 1);
+    s_last = (prev == (int)gridDim.x - 1);
+    if (s_last) {
+      arrive[t] = 0;
+      __threadfence();
+    }
+  }
+  __syncthreads();
+  if (s_last && warp == 0)
+    token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, lane);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
   const moespec_layer_desc &D = *c.desc;
-  size_t smem = (size_t)D.d * sizeof(float);
+  dim3 grid((D.n_experts + 7) / 8, c.M);
+  const Workspace &ws = *c.ws;
   if (D.dtype == MOESPEC_BF16)
-    router_logits_kernel<__nv_bfloat16><<<c.M, 256, smem, c.stream>>>(
-        (const __nv_bfloat16 *)hidden, (const __nv_bfloat16 *)D.router_w, D.router_bias, c.ws->logits,
-        D.n_experts, D.d);
-  else
-    router_logits_kernel<float><<<c.M, 256, smem, c.stream>>>((const float *)hidden, (const float *)D.router_w,
-                                                              D.router_bias, c.ws->logits, D.n_experts, D.d);
-  return cudaGetLastError();
+    return launch_kernel(router_topk_kernel<__nv_bfloat16>, grid, dim3(256), 0, c.stream,
+                         (const __nv_bfloat16 *)hidden, (const __nv_bfloat16 *)D.router_w, D.router_bias, ws.logits,
+                         ws.prob, ws.topk_idx, ws.arrive, D.n_experts, D.d, c.k);
+  return launch_kernel(router_topk_kernel<float>, grid, dim3(256), 0, c.stream, (const float *)hidden,
+                       (const float *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.arrive,
+                       D.n_experts, D.d, c.k);
 }
 
-// ---------------------------------------------------------------------------
-// Warp-wide ranking: repeatedly take the best remaining candidate under
-// (value descending, index ascending).  Lane l owns experts l, l+32, ...
-// `valid` has bit s set when local slot s is still a candidate.  Returns the
-// number of winners written to sel[] (warp-uniform), clears winners from valid.
-// ---------------------------------------------------------------------------
-__device__ __forceinline__ int warp_take_best(const float (&v)[kMaskWords], uint32_t &valid, int rounds,
-                                              int *sel, int lane) {
-  int n = 0;
-  for (int r = 0; r < rounds; ++r) {
-    float bv = -CUDART_INF_F;
-    int bi = 0x7fffffff;
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) {
-      if ((valid >> s) & 1u) {
-        int idx = lane + 32 * s;
-        if (bi == 0x7fffffff || v[s] > bv) { bv = v[s]; bi = idx; }
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-      int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      bool take = (oi != 0x7fffffff) && (bi == 0x7fffffff || ov > bv || (ov == bv && oi < bi));
-      if (take) { bv = ov; bi = oi; }
-    }
-    if (bi == 0x7fffffff) break;
-    if ((bi & 31) == lane) valid &= ~(1u << (bi >> 5));
-    sel[n++] = bi;
-  }
-  return n;
+// Softmax and top-k from caller-supplied logits: one warp per token.
+__global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, double *prob, int *topk_idx, int M,
+                                                           int N, int k) {
+  const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
+  pdl_trigger();
+  pdl_wait();
+  if (t < M) token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, threadIdx.x & 31);
+}
+
+__device__ __forceinline__ double shfl_double(double x, int src) {
+  int lo = __double2loint(x), hi = __double2hiint(x);
+  lo = __shfl_sync(kFull, lo, src);
+  hi = __shfl_sync(kFull, hi, src);
+  return __hiloint2double(hi, lo);
+}
+__device__ __forceinline__ double shfl_xor_double(double x, int mask) {
+  int lo = __double2loint(x), hi = __double2hiint(x);
+  lo = __shfl_xor_sync(kFull, lo, mask);
+  hi = __shfl_xor_sync(kFull, hi, mask);
+  return __hiloint2double(hi, lo);
 }
 
 struct RouteArgs {
@@ -98,213 +209,217 @@ struct RouteArgs {
   long long expert_bytes;       // 3*d*f*sizeof(dtype)
 };
 
+// Re-routing of one token (Eq. 7 / Eq. 8) with its mixing weights (Section 3.3); lane r owns slot r.
+template <int W>
+__device__ __forceinline__ void token_reroute(const RouteArgs &a, int t, int nS, const uint32_t *s_Smask,
+                                              uint32_t *colmask, int mw, int lane) {
+  const Workspace &ws = a.ws;
+  const int N = a.N, k = a.k;
+  int mine = -1;        // kept expert of slot `lane`
+  int base = -1;        // expert whose probability enters the renormalisation sum at position `lane`
+  if (a.policy == MOESPEC_SUBSTITUTION) {
+    uint32_t key[W];
+    uint32_t valid = 0;
+#pragma unroll
+    for (int s = 0; s < W; ++s) {
+      const int idx = lane + 32 * s;
+      key[s] = 0;
+      if (idx < N && ((s_Smask[s] >> lane) & 1u)) {
+        key[s] = order_key(a.logits[(size_t)t * N + idx]);
+        valid |= 1u << s;
+      }
+    }
+    mine = warp_take_best<W>(key, valid, min(k, nS), lane);
+    base = mine;                                   // weights over the constrained selection
+  } else if (lane < k) {
+    const int idx = ws.topk_idx[(size_t)t * k + lane];
+    const bool keep = idx >= 0 && ((s_Smask[idx >> 5] >> (idx & 31)) & 1u);
+    mine = keep ? idx : -1;
+    base = idx;                                    // weights over the original top-k set
+  }
+  const double p_mine = mine >= 0 ? ws.prob[(size_t)t * N + mine] : 0.0;
+  const double p_base = base >= 0 ? (base == mine ? p_mine : ws.prob[(size_t)t * N + base]) : 0.0;
+  double denom = 1.0;
+  if (a.renormalize) {
+    denom = 0.0;
+    for (int r = 0; r < k; ++r) denom += shfl_double(p_base, r);   // rank order
+  }
+  if (lane < k) {
+    ws.assign_idx[(size_t)t * k + lane] = mine;
+    ws.gate_w[(size_t)t * k + lane] = mine >= 0 ? (float)(p_mine / denom) : 0.f;
+    if (mine >= 0) atomicOr(&colmask[(size_t)mine * mw + (t >> 5)], 1u << (t & 31));
+  }
+}
+
 // ---------------------------------------------------------------------------
-// K2: everything between the logits and the expert FFNs, in one CTA.  The data
-// is tiny (M*N <= a few 10k values); one CTA keeps every ranking deterministic
-// and needs no inter-CTA synchronisation.
+// K2: everything between the per-token top-k and the expert FFNs, in one CTA.
+// The data is tiny (M*N <= a few 10k values); one CTA keeps every ranking
+// deterministic and needs no inter-CTA synchronisation.  Dynamic shared memory:
+//   part[nwarps][N]  fp64 partial scores (warp w adds its tokens w, w+32, ... in
+//                    ascending order; the partials are combined in a fixed tree)
+//   colmask[N][mw]   bit t of row i: expert i is in A(t)
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
+  extern __shared__ __align__(16) unsigned char route_smem[];
   __shared__ double s_score[kMaxExperts];
   __shared__ int s_cand[kMaxExperts];
+  __shared__ int s_natcnt[kMaxExperts];
   __shared__ int s_count[kMaxExperts];
   __shared__ int s_offset[kMaxExperts + 1];
   __shared__ int s_unit_base[kMaxExperts + 1];
+  __shared__ int s_Srank[kMaxExperts];
   __shared__ uint32_t s_Smask[kMaskWords];
-  __shared__ int s_nS, s_nactive, s_nunion;
+  __shared__ unsigned long long s_warp_tot[8];
+  __shared__ int s_nS, s_nactive;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const int M = a.M, N = a.N, k = a.k;
-  const int W = kMaskWords;
+  const int mw = (M + 31) >> 5;
   const Workspace &ws = a.ws;
-  uint32_t *natmask = reinterpret_cast<uint32_t *>(ws.natmask);
-  uint32_t *amask = reinterpret_cast<uint32_t *>(ws.amask);
-  if (tid < W) s_Smask[tid] = 0;
+  double *s_part = reinterpret_cast<double *>(route_smem);
+  uint32_t *colmask = reinterpret_cast<uint32_t *>(route_smem + (size_t)nwarps * N * sizeof(double));
+
+#ifdef MOESPEC_ROUTE_TIMING
+  long long tmark[8];
+  int nmark = 0;
+#define ROUTE_MARK() do { if (tid == 0) tmark[nmark++] = clock64(); } while (0)
+#else
+#define ROUTE_MARK() do { } while (0)
+#endif
+  ROUTE_MARK();
+  pdl_trigger();
+  pdl_wait();
+  if (tid < kMaskWords) s_Smask[tid] = 0;
   if (tid == 0) *ws.status = 0;
-
-  // ---- phase A: softmax (Eq. 1) and natural top-k (Eq. 2), one warp per token
-  for (int t = warp; t < M; t += nwarps) {
-    float v[kMaskWords];
-    uint32_t valid = 0;
-    float mx = -CUDART_INF_F;
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) {
-      int idx = lane + 32 * s;
-      v[s] = -CUDART_INF_F;
-      if (idx < N) {
-        v[s] = a.logits[(size_t)t * N + idx];
-        valid |= 1u << s;
-        mx = fmaxf(mx, v[s]);
-      }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    double e[kMaskWords], sum = 0.0;
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) {
-      e[s] = 0.0;
-      if ((valid >> s) & 1u) { e[s] = exp((double)v[s] - (double)mx); sum += e[s]; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s)
-      if ((valid >> s) & 1u) ws.prob[(size_t)t * N + lane + 32 * s] = e[s] / sum;
-
-    int sel[kMaxK];
-    uint32_t rem = valid;
-    int n = warp_take_best(v, rem, k, sel, lane);
-    uint32_t chosen = valid & ~rem;
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) {
-      uint32_t word = __ballot_sync(0xffffffffu, (chosen >> s) & 1u);
-      if (lane == 0) natmask[(size_t)t * W + s] = word;
-    }
-    if (lane == 0)
-      for (int r = 0; r < k; ++r) ws.topk_idx[(size_t)t * k + r] = r < n ? sel[r] : -1;
-  }
+  for (int i = tid; i < N; i += blockDim.x) s_natcnt[i] = 0;
+  for (int i = tid; i < N * mw; i += blockDim.x) colmask[i] = 0;
   __syncthreads();
 
-  // ---- phase B: union (Eq. 3), scores (Eq. 5: tokens added in ascending order, fp64)
-  int my_cand = 0, in_union = 0;
-  if (tid < N) {
-    int natcnt = 0;
-    double s = 0.0;
-    const int w = tid >> 5;
-    const uint32_t bit = 1u << (tid & 31);
-    for (int t = 0; t < M; ++t) {
-      natcnt += (natmask[(size_t)t * W + w] & bit) ? 1 : 0;
-      s += ws.prob[(size_t)t * N + tid];
-    }
-    s_score[tid] = s;
-    ws.score[tid] = s;
-    in_union = natcnt > 0;
-    my_cand = (a.shortlist == MOESPEC_FROM_UNION) ? in_union : 1;
-    s_cand[tid] = my_cand;
+  // ---- phase A: natural counts (Eq. 3) and partial scores (Eq. 5)
+  for (int item = tid; item < M * k; item += blockDim.x) {
+    const int e = ws.topk_idx[item];
+    if (e >= 0) atomicAdd(&s_natcnt[e], 1);
   }
-  const int n_union = __syncthreads_count(in_union);
-  const int n_cand = __syncthreads_count(my_cand);
-  if (tid == 0) s_nunion = n_union;
-  const int nS = min(a.B, n_cand);
+  {
+    double part[kMaskWords];
+#pragma unroll
+    for (int s = 0; s < kMaskWords; ++s) part[s] = 0.0;
+    for (int t = warp; t < M; t += nwarps) {
+#pragma unroll
+      for (int s = 0; s < kMaskWords; ++s)
+        if (lane + 32 * s < N) part[s] += ws.prob[(size_t)t * N + lane + 32 * s];
+    }
+#pragma unroll
+    for (int s = 0; s < kMaskWords; ++s)
+      if (lane + 32 * s < N) s_part[(size_t)warp * N + lane + 32 * s] = part[s];
+  }
+  __syncthreads();
+  ROUTE_MARK();
 
-  // ---- top-B shortlist: rank by counting under (score desc, index asc)
-  if (tid < N && my_cand) {
-    int rank = 0;
-    const double si = s_score[tid];
-    for (int j = 0; j < N; ++j)
+  // ---- phase B: scores (Eq. 5), union (Eq. 3), top-B shortlist by counting under (score desc, index asc)
+  for (int i = warp; i < N; i += nwarps) {
+    double s = lane < nwarps ? s_part[(size_t)lane * N + i] : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += shfl_xor_double(s, o);
+    if (lane == 0) {
+      s_score[i] = s;
+      ws.score[i] = s;
+      s_cand[i] = (a.shortlist == MOESPEC_FROM_UNION) ? (s_natcnt[i] > 0) : 1;
+    }
+  }
+  __syncthreads();
+  const int n_union = __syncthreads_count(tid < N && s_natcnt[tid] > 0);
+  const int n_cand = __syncthreads_count(tid < N && s_cand[tid]);
+  const int nS = min(a.B, n_cand);
+  for (int i = warp; i < N; i += nwarps) {
+    if (!s_cand[i]) continue;
+    const double si = s_score[i];
+    int ahead = 0;
+    for (int j = lane; j < N; j += 32)
       if (s_cand[j]) {
-        double sj = s_score[j];
-        rank += (sj > si || (sj == si && j < tid)) ? 1 : 0;
+        const double sj = s_score[j];
+        ahead += (sj > si || (sj == si && j < i)) ? 1 : 0;
       }
-    if (rank < nS) {
-      ws.S_rank[rank] = tid;
-      atomicOr(&s_Smask[tid >> 5], 1u << (tid & 31));
+    const int rank = __reduce_add_sync(kFull, ahead);
+    if (lane == 0 && rank < nS) {
+      ws.S_rank[rank] = i;
+      s_Srank[rank] = i;
+      atomicOr(&s_Smask[i >> 5], 1u << (i & 31));
     }
   }
   if (tid == 0) s_nS = nS;
   __syncthreads();
+  ROUTE_MARK();
 
   // ---- phase C: re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3), one warp per token
   for (int t = warp; t < M; t += nwarps) {
-    int sel[kMaxK];
-    int n = 0;
-    uint32_t kept_bits = 0;   // local slots of kept experts
-    if (a.policy == MOESPEC_SUBSTITUTION) {
-      float v[kMaskWords];
-      uint32_t valid = 0;
-#pragma unroll
-      for (int s = 0; s < kMaskWords; ++s) {
-        int idx = lane + 32 * s;
-        v[s] = -CUDART_INF_F;
-        if (idx < N && ((s_Smask[s] >> lane) & 1u)) {
-          v[s] = a.logits[(size_t)t * N + idx];
-          valid |= 1u << s;
-        }
-      }
-      uint32_t rem = valid;
-      n = warp_take_best(v, rem, min(k, nS), sel, lane);
-      kept_bits = valid & ~rem;
-      for (int r = n; r < k; ++r) sel[r] = -1;
-    } else {
-      for (int r = 0; r < k; ++r) {
-        int idx = ws.topk_idx[(size_t)t * k + r];
-        bool keep = idx >= 0 && ((s_Smask[idx >> 5] >> (idx & 31)) & 1u);
-        sel[r] = keep ? idx : -1;
-        if (keep && (idx & 31) == lane) kept_bits |= 1u << (idx >> 5);
-      }
-      n = k;
-    }
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) {
-      uint32_t word = __ballot_sync(0xffffffffu, (kept_bits >> s) & 1u);
-      if (lane == 0) amask[(size_t)t * W + s] = word;
-    }
-    if (lane == 0) {
-      double denom = 1.0;
-      if (a.renormalize) {
-        denom = 0.0;
-        if (a.policy == MOESPEC_SUBSTITUTION) {
-          for (int r = 0; r < k; ++r)
-            if (sel[r] >= 0) denom += ws.prob[(size_t)t * N + sel[r]];
-        } else {            // the original top-k set, not the reduced one
-          for (int r = 0; r < k; ++r) {
-            int idx = ws.topk_idx[(size_t)t * k + r];
-            if (idx >= 0) denom += ws.prob[(size_t)t * N + idx];
-          }
-        }
-      }
-      for (int r = 0; r < k; ++r) {
-        ws.assign_idx[(size_t)t * k + r] = sel[r];
-        ws.gate_w[(size_t)t * k + r] = sel[r] >= 0 ? (float)(ws.prob[(size_t)t * N + sel[r]] / denom) : 0.f;
-        ws.tokslot2row[(size_t)t * k + r] = -1;
-      }
-    }
+    if (N <= 32) token_reroute<1>(a, t, nS, s_Smask, colmask, mw, lane);
+    else if (N <= 64) token_reroute<2>(a, t, nS, s_Smask, colmask, mw, lane);
+    else if (N <= 128) token_reroute<4>(a, t, nS, s_Smask, colmask, mw, lane);
+    else token_reroute<8>(a, t, nS, s_Smask, colmask, mw, lane);
   }
   __syncthreads();
+  ROUTE_MARK();
 
-  // ---- phase D: rows per expert and their exclusive scan (Appendix C gather)
-  if (tid < N) {
+  // ---- phase D: rows per expert and exclusive scans of rows, token chunks and active experts
+  {
     int c = 0;
-    const int w = tid >> 5;
-    const uint32_t bit = 1u << (tid & 31);
-    for (int t = 0; t < M; ++t) c += (amask[(size_t)t * W + w] & bit) ? 1 : 0;
-    s_count[tid] = c;
-    ws.count[tid] = c;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int run = 0, na = 0, ub = 0;
-    for (int i = 0; i < N; ++i) {
-      s_offset[i] = run;
-      ws.offset[i] = run;
-      s_unit_base[i] = ub;
-      if (s_count[i] > 0) {
-        ws.active[na++] = i;
-        ub += (s_count[i] + kMaxTokChunk - 1) / kMaxTokChunk;   // token chunks of this expert
+    if (tid < N)
+      for (int w = 0; w < mw; ++w) c += __popc(colmask[(size_t)tid * mw + w]);
+    const int chunks = (c + kMaxTokChunk - 1) / kMaxTokChunk;
+    // rows in bits 0..23, chunks in bits 24..43, active flag in bits 44..
+    unsigned long long v = (unsigned long long)c | ((unsigned long long)chunks << 24) |
+                           ((unsigned long long)(c > 0) << 44);
+    unsigned long long inc = v;
+    if (tid < kMaxExperts) {
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        unsigned long long up = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += up;
       }
-      run += s_count[i];
+      if (lane == 31) s_warp_tot[warp] = inc;
     }
-    s_offset[N] = run;
-    ws.offset[N] = run;
-    s_unit_base[N] = ub;
-    s_nactive = na;
+    __syncthreads();
+    if (tid < kMaxExperts) {
+      unsigned long long pre = inc - v;
+      for (int w = 0; w < warp; ++w) pre += s_warp_tot[w];
+      if (tid < N) {
+        const int row0 = (int)(pre & 0xFFFFFFull), ub = (int)((pre >> 24) & 0xFFFFFull), ai = (int)(pre >> 44);
+        s_count[tid] = c;
+        s_offset[tid] = row0;
+        s_unit_base[tid] = ub;
+        ws.count[tid] = c;
+        ws.offset[tid] = row0;
+        if (c > 0) ws.active[ai] = tid;
+        if (tid == N - 1) {
+          s_offset[N] = row0 + c;
+          ws.offset[N] = row0 + c;
+          s_unit_base[N] = ub + chunks;
+          s_nactive = ai + (c > 0);
+        }
+      }
+    }
   }
   __syncthreads();
+  ROUTE_MARK();
 
-  // ---- phase E: rows ordered by (expert ascending, token ascending)
-  if (tid < N && s_count[tid] > 0) {
-    int row = s_offset[tid];
-    const int w = tid >> 5;
-    const uint32_t bit = 1u << (tid & 31);
-    for (int t = 0; t < M; ++t) {
-      if (amask[(size_t)t * W + w] & bit) {
-        ws.perm_row2tok[row] = t;
-        ws.row2expert[row] = tid;
-        for (int r = 0; r < k; ++r)
-          if (ws.assign_idx[(size_t)t * k + r] == tid) ws.tokslot2row[(size_t)t * k + r] = row;
-        ++row;
-      }
+  // ---- phase E: rows ordered by (expert ascending, token ascending): the row of (t, e) is
+  //      offset[e] + number of tokens below t that were also routed to e
+  for (int item = tid; item < M * k; item += blockDim.x) {
+    const int t = item / k;
+    const int e = ws.assign_idx[item];
+    int row = -1;
+    if (e >= 0) {
+      const uint32_t *cm = colmask + (size_t)e * mw;
+      int below = __popc(cm[t >> 5] & ((1u << (t & 31)) - 1u));
+      for (int w = 0; w < (t >> 5); ++w) below += __popc(cm[w]);
+      row = s_offset[e] + below;
+      ws.perm_row2tok[row] = t;
+      ws.row2expert[row] = e;
     }
+    ws.tokslot2row[item] = row;
   }
+  ROUTE_MARK();
 
   // ---- phase F: tensor-core work units (expert, token chunk, 128-row slab)
   const int n_chunks = s_unit_base[N];
@@ -331,9 +446,9 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
     ws.counters[3] = n_chunks * a.tiles_up;
     ws.counters[4] = n_chunks * a.tiles_down;
     double cov = 0.0;
-    for (int r = 0; r < s_nS; ++r) cov += s_score[ws.S_rank[r]];
+    for (int r = 0; r < s_nS; ++r) cov += s_score[s_Srank[r]];
     moespec_stats st;
-    st.n_union = s_nunion;
+    st.n_union = n_union;
     st.n_shortlist = s_nS;
     st.n_active = s_nactive;
     st.n_rows = R;
@@ -342,10 +457,16 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
     st.coverage = M > 0 ? cov / (double)M : 0.0;
     st.weight_bytes = (long long)s_nactive * a.expert_bytes;
     *ws.stats = st;
+#ifdef MOESPEC_ROUTE_TIMING
+    tmark[nmark++] = clock64();
+    printf("route phases (cycles): A %lld B %lld C %lld D %lld E %lld F+stats %lld total %lld\n", tmark[1] - tmark[0],
+           tmark[2] - tmark[1], tmark[3] - tmark[2], tmark[4] - tmark[3], tmark[5] - tmark[4], tmark[6] - tmark[5],
+           tmark[6] - tmark[0]);
+#endif
   }
 }
 
-cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
+static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) {
   const moespec_layer_desc &D = *c.desc;
   RouteArgs a;
   a.logits = logits;
@@ -356,9 +477,24 @@ cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
   a.tiles_up = tc ? D.f / kTile : 0;
   a.tiles_down = tc ? D.d / kTile : 0;
   a.expert_bytes = 3LL * D.d * D.f * (D.dtype == MOESPEC_BF16 ? 2 : 4);
-  int threads = 1024;
-  route_kernel<<<1, threads, 0, c.stream>>>(a);
-  return cudaGetLastError();
+  const int threads = 1024;
+  const size_t smem = (size_t)(threads / 32) * a.N * sizeof(double) + (size_t)a.N * ((c.M + 31) / 32) * sizeof(uint32_t);
+  if (smem > 40 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+  }
+  return launch_kernel(route_kernel, dim3(1), dim3(threads), smem, c.stream, a);
+}
+
+// Routing after router_topk_kernel has filled logits, prob and topk_idx.
+cudaError_t launch_route_after_router(const LaunchCtx &c) { return launch_route_kernel(c, c.ws->logits); }
+
+// Routing from caller-supplied logits: per-token softmax/top-k first (two launches).
+cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
+  cudaError_t e = launch_kernel(softmax_topk_kernel, dim3((c.M + 3) / 4), dim3(128), 0, c.stream, logits, c.ws->prob,
+                                c.ws->topk_idx, c.M, c.desc->n_experts, c.k);
+  if (e != cudaSuccess) return e;
+  return launch_route_kernel(c, logits);
 }
 
 // ---------------------------------------------------------------------------
@@ -369,6 +505,8 @@ __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restric
                                                           const int *__restrict__ perm,
                                                           const int *__restrict__ counters, int row_vec) {
   const int r = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   if (r >= counters[2]) return;
   const int t = perm[r];
   const uint4 *src = hidden + (size_t)t * row_vec;
@@ -381,9 +519,8 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
   const int row_vec = D.d * (D.dtype == MOESPEC_BF16 ? 2 : 4) / 16;
   const int rows = c.M * c.k;
   if (rows == 0) return cudaSuccess;
-  gather_rows_kernel<<<rows, 128, 0, c.stream>>>((const uint4 *)hidden, (uint4 *)c.ws->x_perm,
-                                                 c.ws->perm_row2tok, c.ws->counters, row_vec);
-  return cudaGetLastError();
+  return launch_kernel(gather_rows_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,
+                       (uint4 *)c.ws->x_perm, (const int *)c.ws->perm_row2tok, (const int *)c.ws->counters, row_vec);
 }
 
 }  // namespace moespec

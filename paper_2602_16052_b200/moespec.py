@@ -14,7 +14,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmoespec.so")
+LIB_PATH = os.environ.get("MOESPEC_LIB") or os.path.join(_HERE, "libmoespec.so")   # override for debug builds
 
 BF16, FP32 = 1, 2
 SUBSTITUTION, TRUNCATION = 1, 2
