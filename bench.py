@@ -319,16 +319,14 @@ def main():
     n_active = [L.get_stats()["n_active"] for L in layers]
     mean_active = sum(n_active) / len(n_active)
     ffn_bytes = mean_active * cfg.expert_weight_bytes()
-    ffn_ms = kt["ffn_gate_up"] + kt["ffn_down"]
+    ffn_ms = kt["ffn"]
     achieved = ffn_bytes / (ffn_ms * 1e-3) / 1e9
     layer_bytes = algorithmic_bytes(cfg, M, mean_active, 4)
     roofline = {
-        "bound": "hbm", "kernel": "ffn_tc_kernel (gate/up launch + down launch)",
+        "bound": "hbm", "kernel": "ffn_tc_kernel (gate/up and down units, one launch)",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
         "traffic": FFN_DRAM_TRAFFIC_BYTES,
         "algorithmic_bytes_per_layer": ffn_bytes, "kernel_us": {n: v * 1e3 for n, v in kt.items()},
-        "gate_up_GBs": mean_active * 2 * cfg.d * cfg.f * 2 / (kt["ffn_gate_up"] * 1e-3) / 1e9,
-        "down_GBs": mean_active * cfg.d * cfg.f * 2 / (kt["ffn_down"] * 1e-3) / 1e9,
         "whole_layer": {"bytes": layer_bytes, "GBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9,
                         "frac": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / peak,
                         "frac_of_nominal_8TBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / 8000.0},

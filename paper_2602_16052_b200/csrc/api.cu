@@ -103,8 +103,9 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.natmask, M * kMaskWords);
   c.take(w.amask, M * kMaskWords);
   c.take(w.arrive, M);
-  c.take(w.units_up, max_chunks * tiles_up);
-  c.take(w.units_down, max_chunks * tiles_down);
+  c.take(w.units, max_chunks * (tiles_up + tiles_down));
+  c.take(w.ready, max_chunks);
+  c.take(w.unit_counter, 4);
   c.take(w.counters, 16);
   c.take(w.stats, 1);
   c.take(w.status, 4);
@@ -143,10 +144,8 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   if (L->use_tc) {
-    for (int phase = 0; phase < 2; ++phase) {
-      if ((e = launch_ffn_tensor_core(c, &L->maps, phase)) != cudaSuccess) return cuda_fail(e);
-      if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
-    }
+    if ((e = launch_ffn_tensor_core(c, &L->maps)) != cudaSuccess) return cuda_fail(e);
+    if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   } else {
     for (int phase = 0; phase < 2; ++phase) {
       if ((e = launch_ffn_cuda_core(c, phase)) != cudaSuccess) return cuda_fail(e);

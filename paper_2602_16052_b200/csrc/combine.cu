@@ -23,6 +23,8 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
   *reinterpret_cast<uint2 *>(p) = raw;
 }
 
+// Grid (M, ceil(d / 1024)): one float4 of one token per thread.  The up-to-k rows of y are all
+// loaded before the first FMA (one memory round trip), then added in slot order.
 template <typename T, typename TO>
 __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ y,
                                                       const float *__restrict__ gate_w,
@@ -30,6 +32,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
                                                       const T *__restrict__ hidden, TO *__restrict__ out, int d,
                                                       int k, int residual) {
   const int t = blockIdx.x;
+  const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
   __shared__ int s_row[kMaxK];
   __shared__ float s_w[kMaxK];
   pdl_trigger();
@@ -39,30 +42,37 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
     s_w[threadIdx.x] = gate_w[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
-  for (int c = threadIdx.x * 4; c < d; c += blockDim.x * 4) {
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = 0; s < k; ++s) {
-      const int row = s_row[s];
-      if (row < 0) continue;
-      const float w = s_w[s];
-      float4 v = load4(y + (size_t)row * d + c);
-      acc.x = fmaf(w, v.x, acc.x);
-      acc.y = fmaf(w, v.y, acc.y);
-      acc.z = fmaf(w, v.z, acc.z);
-      acc.w = fmaf(w, v.w, acc.w);
+  if (c >= d) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < k; s0 += 8) {
+    float4 v[8];
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      const int row = s0 + s < k ? s_row[s0 + s] : -1;
+      v[s] = row >= 0 ? load4(y + (size_t)row * d + c) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
-    if (residual) {
-      float4 h = load4(hidden + (size_t)t * d + c);
-      acc.x += h.x; acc.y += h.y; acc.z += h.z; acc.w += h.w;
+#pragma unroll
+    for (int s = 0; s < 8; ++s) {
+      if (s0 + s < k && s_row[s0 + s] >= 0) {
+        const float w = s_w[s0 + s];
+        acc.x = fmaf(w, v[s].x, acc.x);
+        acc.y = fmaf(w, v[s].y, acc.y);
+        acc.z = fmaf(w, v[s].z, acc.z);
+        acc.w = fmaf(w, v[s].w, acc.w);
+      }
     }
-    store4(out + (size_t)t * d + c, acc);
   }
+  if (residual) {
+    float4 h = load4(hidden + (size_t)t * d + c);
+    acc.x += h.x; acc.y += h.y; acc.z += h.z; acc.w += h.w;
+  }
+  store4(out + (size_t)t * d + c, acc);
 }
 
 template <typename T, typename TO>
 static cudaError_t launch_t(const LaunchCtx &c, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
-  return launch_kernel(combine_kernel<T, TO>, dim3(c.M), dim3(256), 0, c.stream, (const float *)c.ws->y,
+  return launch_kernel(combine_kernel<T, TO>, dim3(c.M, (D.d + 1023) / 1024), dim3(256), 0, c.stream, (const float *)c.ws->y,
                        (const float *)c.ws->gate_w, (const int *)c.ws->tokslot2row, (const T *)hidden, (TO *)out, D.d,
                        c.k, D.residual);
 }

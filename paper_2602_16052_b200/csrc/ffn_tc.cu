@@ -6,14 +6,24 @@
 // routed token rows are the B operand (N axis, padded to a multiple of 32),
 // fp32 accumulators live in tensor memory.
 //
-//   phase 0 (gate/up):  D_g = W1[e, slab, :] X_e^T,  D_u = W3[e, slab, :] X_e^T,
-//                       h_mid[row, slab] = bf16(silu(D_g) * D_u)
-//   phase 1 (down):     D = W2[e, slab, :] H_e^T,     y[row, slab] = D  (fp32)
+//   gate/up unit:  D_g = W1[e, slab, :] X_e^T,  D_u = W3[e, slab, :] X_e^T,
+//                  h_mid[row, slab] = bf16(silu(D_g) * D_u)
+//   down unit:     D = W2[e, slab, :] H_e^T,     y[row, slab] = D  (fp32)
 //
-// One persistent CTA per SM, six warps:
-//   warp 0  lane 0: TMA producer.  Streams 64-wide K chunks of the weight slab(s)
-//                   (3-D tensor map, expert id is the outer coordinate: no
-//                   stacking copy) and of the token rows into a ring of stages.
+// One launch covers both kinds.  The unit list holds every gate/up unit, then
+// every down unit; persistent CTAs (one per SM) draw units in list order from a
+// global dispenser, so the gate/up tail overlaps the start of the down
+// projection.  A down unit needs all of its expert chunk's h_mid: each finished
+// gate/up unit bumps a per-chunk ready counter (release), and the producer of a
+// down unit waits (bounded, acquire) for the counter to reach the slab count.
+// Units are handed out in order and gate/up units never wait, so every unit a
+// down unit waits for is already running or done: there is no circular wait.
+//
+// Six warps per CTA:
+//   warp 0  lane 0: dispenser + TMA producer.  Streams 64-wide K chunks of the
+//                   weight slab(s) (3-D tensor map, expert id is the outer
+//                   coordinate: no stacking copy) and of the token rows into a
+//                   ring of stages, 32 KB of weights per stage.
 //   warp 1  lane 0: issues tcgen05.mma (kind::f16, M=128, N=n_pad, K=16) from the
 //                   stage's swizzled shared memory into TMEM; tcgen05.commit frees
 //                   the stage and finally publishes the accumulator.
@@ -34,21 +44,28 @@ constexpr int kABytes = kTile * kChunkK * 2;     // 16 KB: one weight slab chunk
 constexpr int kBOffset = 2 * kABytes;            // token rows start after two weight chunks
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
-constexpr int kCtrlBytes = 256;                  // barriers + TMEM base + abort flag
+constexpr int kCtrlBytes = 512;                  // barriers, unit queue, TMEM base, abort flag
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kSpinLimitCycles = 2000000000LL;   // ~1 s at 2 GHz
 
+constexpr int kQueue = 4;                        // units in flight between the producer and its consumers
+
 struct TcArgs {
   const Unit *units;
-  const int *n_units;
-  int phase;            // 0 gate/up, 1 down
-  int k_iters;          // ring stages per unit: K/64 in phase 0 (gate chunk + up chunk), K/128 in phase 1
-  int b1_off;           // phase 1: offset of the second token slab inside a stage
+  const int *n_units;   // [0] gate/up units, [1] down units
+  int *unit_counter;    // dispenser
+  int *ready;           // per (expert, token chunk): finished gate/up units
+  int tiles_up;         // gate/up units per chunk = value of ready[] that releases its down units
+  int k_iters_up;       // ring stages per gate/up unit: d / 64 (one K chunk of gate and of up per stage)
+  int k_iters_down;     // ring stages per down unit: f / 128 (two K chunks) or f / 64 (one)
+  int down_double;      // 1: a down stage carries two K chunks
+  int b1_off;           // offset of the second token slab inside a stage
   int n_stages;
   int stage_bytes;
   int acc_bufs;         // 1 or 2 accumulator buffers of 256 TMEM columns
-  void *out;            // h_mid (bf16) or y (fp32)
-  int out_ld;           // f or d
+  __nv_bfloat16 *h_mid; // [R, f]
+  float *y;             // [R, d]
+  int f, d;
   int *status;
 };
 
@@ -148,6 +165,14 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
 
 }  // namespace
 
+__device__ __forceinline__ int ld_acquire(const int *p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // stages first (1024-byte aligned for the 128-byte swizzle), control block after
@@ -159,8 +184,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   const uint32_t bar_empty = ctrl + 8 * kMaxStages;     // [kMaxStages]
   const uint32_t bar_acc_full = ctrl + 16 * kMaxStages; // [2]
   const uint32_t bar_acc_empty = bar_acc_full + 16;     // [2]
-  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + 16 * kMaxStages + 32);
-  volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + 16 * kMaxStages + 36);
+  const uint32_t bar_q_full = bar_acc_empty + 16;       // [kQueue]
+  const uint32_t bar_q_empty = bar_q_full + 8 * kQueue; // [kQueue]
+  constexpr int kMiscOff = 16 * kMaxStages + 32 + 16 * kQueue;   // 224
+  volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + kMiscOff);
+  volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + kMiscOff + 4);
+  Unit *q_unit = reinterpret_cast<Unit *>(ctrl_gen + 256);       // [kQueue] x 32 bytes
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_stages = a.n_stages;
@@ -174,6 +203,10 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_acc_full + 8 * b, 1);
       mbar_init(bar_acc_empty + 8 * b, 128);
+    }
+    for (int q = 0; q < kQueue; ++q) {
+      mbar_init(bar_q_full + 8 * q, 1);
+      mbar_init(bar_q_empty + 8 * q, 129);      // the MMA thread and the 128 epilogue threads
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -191,42 +224,68 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   const uint32_t tmem_base = *tmem_slot;
   // everything above overlaps the tail of the previous kernel; its results are read from here on
   pdl_wait();
-  const int n_units = *a.n_units;
-
-  const CUtensorMap *map_a0 = a.phase == 0 ? &maps.w_gate : &maps.w_down;
-  const CUtensorMap *map_a1 = &maps.w_up;
-  const CUtensorMap *map_b = a.phase == 0 ? &maps.x_perm : &maps.h_mid;
-  // every stage carries 32 KB of weights: phase 0 one K chunk of gate and of up, phase 1 two K chunks of down
-  const uint32_t b_slabs = a.phase == 0 ? 1u : 2u;
 
   if (warp == 0 && lane == 0) {
-    // ===================================================== TMA producer
-    uint32_t it = 0;
+    // ===================================================== dispenser + TMA producer
+    const int n_up = a.n_units[0], n_total = n_up + a.n_units[1];
+    uint32_t it = 0, qi = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-      const Unit un = a.units[u];
+    int u = atomicAdd(a.unit_counter, 1);
+    while (ok) {
+      const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
+      if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag)) { ok = false; break; }
+      Unit un;
+      if (u < n_total) {
+        un = a.units[u];
+      } else {
+        un.expert = -1; un.tile = 0; un.row0 = 0; un.n_rows = 0; un.chunk = 0; un.phase = 0; un.pad0 = 0; un.pad1 = 0;
+      }
+      q_unit[q] = un;
+      mbar_arrive(bar_q_full + 8 * q);          // release: the queue slot is visible to the consumers
+      ++qi;
+      if (un.expert < 0) break;
+      const int u_next = atomicAdd(a.unit_counter, 1);   // in flight while this unit streams
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
-      for (int kc = 0; kc < a.k_iters; ++kc, ++it) {
+      if (un.phase == 1) {
+        // the rows of h_mid this unit reads are complete once every gate/up slab of the chunk is done
+        const long long t0 = clock64();
+        while (ld_acquire(a.ready + un.chunk) < a.tiles_up) {
+          if (*abort_flag || clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; ok = false; break; }
+          __nanosleep(64);
+        }
+        if (!ok) break;
+        fence_proxy_async();                    // order the acquire before the TMA reads of h_mid
+      }
+      const int k_iters = un.phase == 0 ? a.k_iters_up : a.k_iters_down;
+      const CUtensorMap *map_b = un.phase == 0 ? &maps.x_perm : &maps.h_mid;
+      for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t full = bar_full + 8 * s;
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
-        mbar_expect_tx(full, 2u * kABytes + b_slabs * (uint32_t)n_pad * 128u);
-        if (a.phase == 0) {
-          tma_load_3d(stage, map_a0, full, kc * kChunkK, un.tile * kTile, un.expert);
-          tma_load_3d(stage + kABytes, map_a1, full, kc * kChunkK, un.tile * kTile, un.expert);
+        if (un.phase == 0) {
+          mbar_expect_tx(full, 2u * kABytes + (uint32_t)n_pad * 128u);
+          tma_load_3d(stage, &maps.w_gate, full, kc * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage + kABytes, &maps.w_up, full, kc * kChunkK, un.tile * kTile, un.expert);
           for (int b = 0; b < n_pad / kTokBox; ++b)
             tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
-        } else {
-          tma_load_3d(stage, map_a0, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert);
-          tma_load_3d(stage + kABytes, map_a0, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert);
+        } else if (a.down_double) {
+          mbar_expect_tx(full, 2u * kABytes + 2u * (uint32_t)n_pad * 128u);
+          tma_load_3d(stage, &maps.w_down, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage + kABytes, &maps.w_down, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert);
           for (int b = 0; b < n_pad / kTokBox; ++b) {
             tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, (2 * kc) * kChunkK, un.row0 + b * kTokBox);
             tma_load_2d(stage + a.b1_off + b * (kTokBox * 128), map_b, full, (2 * kc + 1) * kChunkK,
                         un.row0 + b * kTokBox);
           }
+        } else {
+          mbar_expect_tx(full, (uint32_t)kABytes + (uint32_t)n_pad * 128u);
+          tma_load_3d(stage, &maps.w_down, full, kc * kChunkK, un.tile * kTile, un.expert);
+          for (int b = 0; b < n_pad / kTokBox; ++b)
+            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
         }
       }
+      u = u_next;
     }
     if (!ok) {
       // drain: wait (bounded) until every copy this thread issued has landed
@@ -239,22 +298,27 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     }
   } else if (warp == 1 && lane == 0) {
     // ===================================================== MMA issuer
-    uint32_t it = 0, acc_it = 0;
+    uint32_t it = 0, acc_it = 0, qi = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
-      const Unit un = a.units[u];
+    while (ok) {
+      const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
+      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag)) break;
+      const Unit un = q_unit[q];
+      ++qi;
+      if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t idesc = instr_desc_bf16(n_pad);
       const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
-      if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) break;
       tc_fence_after();
       const uint32_t tmem_d = tmem_base + ab * 256u;
-      for (int kc = 0; kc < a.k_iters; ++kc, ++it) {
+      const int k_iters = un.phase == 0 ? a.k_iters_up : a.k_iters_down;
+      for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
-        if (a.phase == 0) {
+        if (un.phase == 0) {
 #pragma unroll
           for (int kk = 0; kk < kChunkK / 16; ++kk) {
             const uint32_t acc = (kc > 0 || kk > 0) ? 1u : 0u;
@@ -263,8 +327,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             tc_mma_bf16(tmem_d + (uint32_t)n_pad, smem_desc_sw128(stage + kABytes + kk * 32), bdesc, idesc, acc);
           }
         } else {
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
+          const int halves = a.down_double ? 2 : 1;
+          for (int half = 0; half < halves; ++half) {
             const uint32_t a_off = stage + half * kABytes;
             const uint32_t b_off = stage + (half ? (uint32_t)a.b1_off : (uint32_t)kBOffset);
 #pragma unroll
@@ -275,48 +339,61 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         }
         tc_commit(bar_empty + 8 * s);      // stage reusable once these MMAs have read it
       }
-      if (ok) tc_commit(bar_acc_full + 8 * ab);
+      if (!ok) break;
+      tc_commit(bar_acc_full + 8 * ab);
+      mbar_arrive(bar_q_empty + 8 * q);
+      ++acc_it;
     }
   } else if (warp >= 2) {
     // ===================================================== epilogue
     const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 belong to this warp
     const int row_in_tile = quarter * 32 + lane;
-    uint32_t acc_it = 0;
-    bool ok = true;
-    for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
-      const Unit un = a.units[u];
+    uint32_t acc_it = 0, qi = 0;
+    while (true) {
+      const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
+      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag)) break;
+      const Unit un = q_unit[q];
+      ++qi;
+      if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
-      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag)) { ok = false; break; }
+      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag)) break;
       tc_fence_after();
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
-      const int col_out = un.tile * kTile + row_in_tile;    // index along f (phase 0) or d (phase 1)
+      const int col_out = un.tile * kTile + row_in_tile;    // index along f (gate/up) or d (down)
       for (int c0 = 0; c0 < un.n_rows; c0 += 16) {
         uint32_t g[16];
         tc_ld16(taddr + c0, g);
-        if (a.phase == 0) {
+        if (un.phase == 0) {
           uint32_t up[16];
           tc_ld16(taddr + n_pad + c0, up);
           tc_ld_wait();
-          __nv_bfloat16 *out = reinterpret_cast<__nv_bfloat16 *>(a.out);
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             if (c0 + i < un.n_rows) {
               const float gv = __uint_as_float(g[i]), uv = __uint_as_float(up[i]);
               const float m = gv / (1.f + __expf(-gv)) * uv;
-              out[(size_t)(un.row0 + c0 + i) * a.out_ld + col_out] = __float2bfloat16_rn(m);
+              a.h_mid[(size_t)(un.row0 + c0 + i) * a.f + col_out] = __float2bfloat16_rn(m);
             }
           }
         } else {
           tc_ld_wait();
-          float *out = reinterpret_cast<float *>(a.out);
 #pragma unroll
           for (int i = 0; i < 16; ++i)
-            if (c0 + i < un.n_rows) out[(size_t)(un.row0 + c0 + i) * a.out_ld + col_out] = __uint_as_float(g[i]);
+            if (c0 + i < un.n_rows) a.y[(size_t)(un.row0 + c0 + i) * a.d + col_out] = __uint_as_float(g[i]);
         }
       }
       tc_fence_before();
       mbar_arrive(bar_acc_empty + 8 * ab);
+      if (un.phase == 0) {
+        // publish this slab of h_mid: every thread's stores are fenced, then one thread bumps the counter
+        __threadfence();
+        fence_proxy_async();
+        epilogue_bar();
+        if (threadIdx.x == 64) atomicAdd(a.ready + un.chunk, 1);
+      }
+      mbar_arrive(bar_q_empty + 8 * q);
+      ++acc_it;
     }
   }
 
@@ -389,32 +466,30 @@ static int sm_count_cached(int device) {
   return n;
 }
 
-cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, int phase) {
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps) {
   const moespec_layer_desc &D = *c.desc;
   const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
   TcArgs a;
-  a.phase = phase;
+  a.down_double = n_pad_max <= 128 ? 1 : 0;      // two K chunks per down stage while both token slabs fit
   a.b1_off = kBOffset + n_pad_max * 128;
-  a.stage_bytes = kBOffset + (phase == 0 ? 1 : 2) * n_pad_max * 128;
+  a.stage_bytes = kBOffset + (a.down_double ? 2 : 1) * n_pad_max * 128;
   int stages = (kSmemBudget - 1024 - kCtrlBytes) / a.stage_bytes;
   a.n_stages = stages > kMaxStages ? kMaxStages : stages;
   a.acc_bufs = 2 * n_pad_max <= 256 ? 2 : 1;
   a.status = c.ws->status;
+  a.units = c.ws->units;
+  a.n_units = c.ws->counters + 3;
+  a.unit_counter = c.ws->unit_counter;
+  a.ready = c.ws->ready;
+  a.tiles_up = D.f / kTile;
+  a.k_iters_up = D.d / kChunkK;
+  a.k_iters_down = a.down_double ? D.f / (2 * kChunkK) : D.f / kChunkK;
+  a.h_mid = reinterpret_cast<__nv_bfloat16 *>(c.ws->h_mid);
+  a.y = c.ws->y;
+  a.f = D.f;
+  a.d = D.d;
   const int grid = sm_count_cached(D.device);
   const size_t smem = (size_t)a.n_stages * a.stage_bytes + 1024 + kCtrlBytes;
-  if (phase == 0) {
-    a.units = c.ws->units_up;
-    a.n_units = c.ws->counters + 3;
-    a.k_iters = D.d / kChunkK;
-    a.out = c.ws->h_mid;
-    a.out_ld = D.f;
-  } else {
-    a.units = c.ws->units_down;
-    a.n_units = c.ws->counters + 4;
-    a.k_iters = D.f / (2 * kChunkK);
-    a.out = c.ws->y;
-    a.out_ld = D.d;
-  }
   return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, *maps, a);
 }
 

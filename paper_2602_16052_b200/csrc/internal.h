@@ -17,11 +17,14 @@ constexpr int kMaxTokChunk = 256;          // tokens per work unit (MMA N limit)
 
 // One tensor-core work unit: a 128-row slab of one expert's weight matrix
 // against one chunk (<= 256) of that expert's routed rows.
-struct Unit {
+struct __align__(16) Unit {
   int expert;
   int tile;       // slab index along f (gate/up phase) or d (down phase)
   int row0;       // first routed row of the chunk
   int n_rows;     // rows in the chunk (1..256)
+  int chunk;      // global index of the (expert, token chunk) pair: indexes the ready counters
+  int phase;      // 0 gate/up, 1 down
+  int pad0, pad1;
 };
 
 // Device-resident routing state and scratch of one layer handle.
@@ -42,8 +45,9 @@ struct Workspace {
   unsigned *natmask;    // [max_M, 8] bit i of row t: expert i in T_k(h_t)
   unsigned *amask;      // [max_M, 8] bit i of row t: expert i in A(t)
   int *arrive;          // [max_M] per-token arrival counters of router_topk_kernel (zero between calls)
-  Unit *units_up;       // gate/up units
-  Unit *units_down;     // down units
+  Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
+  int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
+  int *unit_counter;    // next unit to hand out; zeroed by the route kernel
   int *counters;        // [0]=n_S [1]=n_active [2]=R [3]=n_units_up [4]=n_units_down
   moespec_stats *stats; // device copy
   int *status;          // device status word (0 = ok)
@@ -105,7 +109,7 @@ struct TcMaps {
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes
-cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, int phase);   // 0 gate/up, 1 down
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps);   // both phases, one launch
 // combine.cu
 cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out);
 

@@ -101,18 +101,20 @@ __device__ __forceinline__ void token_phase(const float *zrow, int N, int k, dou
 
 // ---------------------------------------------------------------------------
 // K1: z[t,i] = b_i + w_i . h_t with fp32 accumulation, fused with the token's
-// softmax and top-k.  Grid (ceil(N/8), M): one warp per (token, expert) pair;
-// both rows are read with 16-byte loads issued before the first FMA.  Each CTA
-// then bumps the token's arrival counter; the CTA that sees the final count
-// finishes the token and resets the counter for the next call.
+// softmax and top-k.  A CTA takes TT tokens x 8 experts; warp w owns expert w of
+// the tile, keeps 2 KB chunks of its router row in registers and runs them
+// against the TT token rows (shared through L1), so a router row is read once per
+// token tile.  Each CTA then bumps the token tile's arrival counter; the CTA
+// that sees the final count runs softmax and top-k of those TT tokens (one warp
+// each) and resets the counter for the next call.  A counter, never a wait.
 // ---------------------------------------------------------------------------
-template <typename T>
+template <typename T, int TT>
 __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                           const float *__restrict__ bias, float *logits,
-                                                          double *prob, int *topk_idx, int *arrive, int N, int d,
-                                                          int k) {
+                                                          double *prob, int *topk_idx, int *arrive, int M, int N,
+                                                          int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.y;
+  const int t0 = blockIdx.y * TT;
   const int i = blockIdx.x * 8 + warp;
   __shared__ int s_last;
   pdl_trigger();
@@ -120,62 +122,76 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   if (i < N) {
     constexpr int VEC = 16 / sizeof(T);
     constexpr int U = 8;
-    const T *h = hidden + (size_t)t * d;
     const T *w = Wr + (size_t)i * d;
-    float acc = 0.f;
+    float acc[TT];
+#pragma unroll
+    for (int tt = 0; tt < TT; ++tt) acc[tt] = 0.f;
     for (int j0 = lane * VEC; j0 < d; j0 += 32 * VEC * U) {
-      uint4 rw[U], rh[U];
+      uint4 rw[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int j = j0 + u * 32 * VEC;
-        if (j < d) {
-          rw[u] = *reinterpret_cast<const uint4 *>(w + j);
-          rh[u] = *reinterpret_cast<const uint4 *>(h + j);
-        }
-      }
+      for (int u = 0; u < U; ++u)
+        if (j0 + u * 32 * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(w + j0 + u * 32 * VEC);
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int j = j0 + u * 32 * VEC;
-        if (j < d) {
-          const T *ew = reinterpret_cast<const T *>(&rw[u]);
-          const T *eh = reinterpret_cast<const T *>(&rh[u]);
+      for (int tt = 0; tt < TT; ++tt) {
+        if (t0 + tt >= M) break;
+        const T *h = hidden + (size_t)(t0 + tt) * d;
+        uint4 rh[U];
 #pragma unroll
-          for (int v = 0; v < VEC; ++v) acc = fmaf(to_float(ew[v]), to_float(eh[v]), acc);
+        for (int u = 0; u < U; ++u)
+          if (j0 + u * 32 * VEC < d) rh[u] = *reinterpret_cast<const uint4 *>(h + j0 + u * 32 * VEC);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (j0 + u * 32 * VEC < d) {
+            const T *ew = reinterpret_cast<const T *>(&rw[u]);
+            const T *eh = reinterpret_cast<const T *>(&rh[u]);
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) acc[tt] = fmaf(to_float(ew[v]), to_float(eh[v]), acc[tt]);
+          }
         }
       }
     }
+    const float b = bias ? bias[i] : 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFull, acc, o);
-    if (lane == 0) {
-      logits[(size_t)t * N + i] = acc + (bias ? bias[i] : 0.f);
-      __threadfence();
+    for (int tt = 0; tt < TT; ++tt) {
+      float a = acc[tt];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(kFull, a, o);
+      if (lane == 0 && t0 + tt < M) logits[(size_t)(t0 + tt) * N + i] = a + b;
     }
+    if (lane == 0) __threadfence();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int prev = atomicAdd(&arrive[t], 1);
+    const int prev = atomicAdd(&arrive[blockIdx.y], 1);
     s_last = (prev == (int)gridDim.x - 1);
     if (s_last) {
-      arrive[t] = 0;
+      arrive[blockIdx.y] = 0;
       __threadfence();
     }
   }
   __syncthreads();
-  if (s_last && warp == 0)
+  if (s_last && warp < TT && t0 + warp < M) {
+    const int t = t0 + warp;
     token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, lane);
+  }
+}
+
+template <typename T>
+static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
+  const moespec_layer_desc &D = *c.desc;
+  const Workspace &ws = *c.ws;
+  const int ex_tiles = (D.n_experts + 7) / 8;
+  if (c.M <= 64)
+    return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
+                         (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
+                         ws.arrive, c.M, D.n_experts, D.d, c.k);
+  return launch_kernel(router_topk_kernel<T, 8>, dim3(ex_tiles, (c.M + 7) / 8), dim3(256), 0, c.stream,
+                       (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
+                       ws.arrive, c.M, D.n_experts, D.d, c.k);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
-  const moespec_layer_desc &D = *c.desc;
-  dim3 grid((D.n_experts + 7) / 8, c.M);
-  const Workspace &ws = *c.ws;
-  if (D.dtype == MOESPEC_BF16)
-    return launch_kernel(router_topk_kernel<__nv_bfloat16>, grid, dim3(256), 0, c.stream,
-                         (const __nv_bfloat16 *)hidden, (const __nv_bfloat16 *)D.router_w, D.router_bias, ws.logits,
-                         ws.prob, ws.topk_idx, ws.arrive, D.n_experts, D.d, c.k);
-  return launch_kernel(router_topk_kernel<float>, grid, dim3(256), 0, c.stream, (const float *)hidden,
-                       (const float *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.arrive,
-                       D.n_experts, D.d, c.k);
+  return c.desc->dtype == MOESPEC_BF16 ? launch_router_t<__nv_bfloat16>(c, hidden) : launch_router_t<float>(c, hidden);
 }
 
 // Softmax and top-k from caller-supplied logits: one warp per token.
@@ -286,9 +302,14 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
 #else
 #define ROUTE_MARK() do { } while (0)
 #endif
-  ROUTE_MARK();
   pdl_trigger();
   pdl_wait();
+#ifdef MOESPEC_ROUTE_TIMING
+  for (int rep = 0; rep < 2; ++rep) {
+  nmark = 0;
+  __syncthreads();
+#endif
+  ROUTE_MARK();
   if (tid < kMaskWords) s_Smask[tid] = 0;
   if (tid == 0) *ws.status = 0;
   for (int i = tid; i < N; i += blockDim.x) s_natcnt[i] = 0;
@@ -421,9 +442,13 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
   }
   ROUTE_MARK();
 
-  // ---- phase F: tensor-core work units (expert, token chunk, 128-row slab)
+  // ---- phase F: tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all
+  //      down units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
   const int n_chunks = s_unit_base[N];
   if (a.tiles_up > 0) {
+    const int n_up = n_chunks * a.tiles_up;
+    for (int i = tid; i < n_chunks; i += blockDim.x) ws.ready[i] = 0;
+    if (tid == 0) *ws.unit_counter = 0;
     for (int i = warp; i < N; i += nwarps) {
       const int cnt = s_count[i];
       if (cnt == 0) continue;
@@ -432,8 +457,10 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
         const int row0 = s_offset[i] + c * kMaxTokChunk;
         const int rows = min(kMaxTokChunk, cnt - c * kMaxTokChunk);
         const int ci = s_unit_base[i] + c;
-        for (int tl = lane; tl < a.tiles_up; tl += 32) ws.units_up[(size_t)ci * a.tiles_up + tl] = Unit{i, tl, row0, rows};
-        for (int tl = lane; tl < a.tiles_down; tl += 32) ws.units_down[(size_t)ci * a.tiles_down + tl] = Unit{i, tl, row0, rows};
+        for (int tl = lane; tl < a.tiles_up; tl += 32)
+          ws.units[(size_t)ci * a.tiles_up + tl] = Unit{i, tl, row0, rows, ci, 0, 0, 0};
+        for (int tl = lane; tl < a.tiles_down; tl += 32)
+          ws.units[(size_t)n_up + (size_t)ci * a.tiles_down + tl] = Unit{i, tl, row0, rows, ci, 1, 0, 0};
       }
     }
   }
@@ -464,6 +491,10 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
            tmark[6] - tmark[0]);
 #endif
   }
+#ifdef MOESPEC_ROUTE_TIMING
+  __syncthreads();
+  }
+#endif
 }
 
 static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) {

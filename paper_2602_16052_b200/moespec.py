@@ -240,7 +240,8 @@ class Layer:
         _check(lib().moespec_get_stats(self._h, C.byref(st)), "moespec_get_stats")
         return st.as_dict()
 
-    KERNEL_NAMES = ("router_logits", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
+    KERNEL_NAMES_TC = ("router_topk", "route", "gather", "ffn", "combine")
+    KERNEL_NAMES_CC = ("router_topk", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
 
     def set_profiling(self, on: bool):
         _check(lib().moespec_set_profiling(self._h, int(on)), "moespec_set_profiling")
@@ -251,7 +252,8 @@ class Layer:
         n = C.c_int(0)
         _check(lib().moespec_get_kernel_times(self._h, C.cast(ms, C.c_void_p), 8, C.cast(C.byref(n), C.c_void_p)),
                "moespec_get_kernel_times")
-        return {self.KERNEL_NAMES[i]: float(ms[i]) for i in range(min(n.value, len(self.KERNEL_NAMES)))}
+        names = self.KERNEL_NAMES_TC if n.value == len(self.KERNEL_NAMES_TC) else self.KERNEL_NAMES_CC
+        return {names[i]: float(ms[i]) for i in range(min(n.value, len(names)))}
 
     def last_launch_count(self) -> int:
         return lib().moespec_last_launch_count(self._h)
