@@ -153,9 +153,9 @@ int moespec_route_from_logits(moespec_layer_t *layer, const float *logits, int M
  * fields of moespec_layer_desc.  Enqueues on `stream` and returns.
  *
  * Sharing: all calls in the process use the same scratch array, which keeps the
- * previous call's contents; the kernel rewrites every word before reading it,
- * so nothing needs clearing, but two calls that overlap on the GPU (different
- * streams or threads) race on it.  Serialise them.
+ * previous call's contents; each call first clears, on its stream, the part the
+ * kernels accumulate into.  Two calls that overlap on the GPU (different streams
+ * or threads) race on the array.  Serialise them.
  *
  * First call: the first call on each device looks up the array's device address
  * (cudaGetSymbolAddress) with that device current; make that first call before

@@ -100,9 +100,13 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.perm_row2tok, (size_t)R_cap);
   c.take(w.row2expert, (size_t)R_cap);
   c.take(w.tokslot2row, M * K);
-  c.take(w.natmask, M * kMaskWords);
-  c.take(w.amask, M * kMaskWords);
+  w.mask_words = (int)((M + 31) / 32);
+  c.take(w.score_fx, N);
+  c.take(w.natcnt_acc, N);
+  c.take(w.count_acc, N);
+  c.take(w.colmask, N * (size_t)w.mask_words);
   c.take(w.arrive, M);
+  c.take(w.arrive_route, 4);
   c.take(w.units, max_chunks * (tiles_up + tiles_down));
   c.take(w.ready, max_chunks);
   c.take(w.unit_counter, 4);

@@ -42,9 +42,15 @@ struct Workspace {
   int *perm_row2tok;    // [R_cap]
   int *row2expert;      // [R_cap]
   int *tokslot2row;     // [max_M, max_k]
-  unsigned *natmask;    // [max_M, 8] bit i of row t: expert i in T_k(h_t)
-  unsigned *amask;      // [max_M, 8] bit i of row t: expert i in A(t)
-  int *arrive;          // [max_M] per-token arrival counters of router_topk_kernel (zero between calls)
+  // accumulators shared by the CTAs of one call; every one of them is zero between calls (the routing
+  // kernel's last CTA clears what the call used)
+  unsigned long long *score_fx;  // [N] sum_t g_i(h_t) in 2^-52 fixed point: exact integer adds, any order
+  int *natcnt_acc;      // [N] number of tokens with expert i in T_k(h_t)
+  int *count_acc;       // [N] number of tokens with expert i in A(t)
+  unsigned *colmask;    // [N, ceil(max_M/32)] bit t of row i: expert i in A(t)
+  int *arrive;          // [max_M] arrival counters of router_topk_kernel's token tiles
+  int *arrive_route;    // [1] arrival counter of route_kernel's CTAs
+  int mask_words;       // ceil(max_M / 32)
   Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
   int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
   int *unit_counter;    // next unit to hand out; zeroed by the route kernel

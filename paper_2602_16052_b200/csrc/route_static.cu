@@ -10,9 +10,10 @@
 // that array (kRouteStaticScratchBytes) until the process exits.
 //
 // The array is shared by every call in the process and keeps the previous
-// call's contents.  The routing kernel writes every scratch word before it
-// reads it, so nothing has to be cleared between calls; two calls that overlap
-// on the GPU (different streams, or different threads) would race on it.
+// call's contents.  The accumulators the routing kernels add into are cleared
+// on the caller's stream at the start of every call; everything else is written
+// before it is read.  Two calls that overlap on the GPU (different streams, or
+// different threads) would race on the array.
 #include "internal.h"
 
 #include <mutex>
@@ -28,13 +29,20 @@ constexpr int kStaticMaxRows = MOESPEC_ROUTE_STATIC_MAX_ROWS;
 
 constexpr size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 constexpr size_t kOffProb = 0;                                                              // double [M, N]
-constexpr size_t kOffNat = kOffProb + align256(sizeof(double) * kStaticMaxM * kStaticMaxN); // uint [M, 8]
-constexpr size_t kOffAmask = kOffNat + align256(sizeof(unsigned) * kStaticMaxM * kMaskWords);
-constexpr size_t kOffActive = kOffAmask + align256(sizeof(unsigned) * kStaticMaxM * kMaskWords);
+constexpr size_t kOffActive = kOffProb + align256(sizeof(double) * kStaticMaxM * kStaticMaxN);
 constexpr size_t kOffRow2Exp = kOffActive + align256(sizeof(int) * kStaticMaxN);
 constexpr size_t kOffStats = kOffRow2Exp + align256(sizeof(int) * kStaticMaxRows);
 constexpr size_t kOffStatus = kOffStats + align256(sizeof(moespec_stats));
-constexpr size_t kRouteStaticScratchBytes = kOffStatus + 256;
+// accumulators that must be zero when a call starts (cleared on the stream before every call)
+constexpr size_t kOffZero = kOffStatus + 256;
+constexpr int kStaticMaskWords = (kStaticMaxM + 31) / 32;
+constexpr size_t kOffScoreFx = kOffZero;                                                    // ull [N]
+constexpr size_t kOffNatcnt = kOffScoreFx + align256(sizeof(unsigned long long) * kStaticMaxN);
+constexpr size_t kOffCountAcc = kOffNatcnt + align256(sizeof(int) * kStaticMaxN);
+constexpr size_t kOffColmask = kOffCountAcc + align256(sizeof(int) * kStaticMaxN);         // uint [N, mask words]
+constexpr size_t kOffArrive = kOffColmask + align256(sizeof(unsigned) * kStaticMaxN * kStaticMaskWords);
+constexpr size_t kRouteStaticScratchBytes = kOffArrive + 256;
+constexpr size_t kZeroBytes = kRouteStaticScratchBytes - kOffZero;
 
 // In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
 static __device__ __align__(256) unsigned char g_route_scratch[kRouteStaticScratchBytes];
@@ -83,8 +91,15 @@ extern "C" int moespec_route_static(const float *logits, int M, int N, int k, in
 
   Workspace ws{};
   ws.prob = reinterpret_cast<double *>(scratch + kOffProb);
-  ws.natmask = reinterpret_cast<unsigned *>(scratch + kOffNat);
-  ws.amask = reinterpret_cast<unsigned *>(scratch + kOffAmask);
+  ws.score_fx = reinterpret_cast<unsigned long long *>(scratch + kOffScoreFx);
+  ws.natcnt_acc = reinterpret_cast<int *>(scratch + kOffNatcnt);
+  ws.count_acc = reinterpret_cast<int *>(scratch + kOffCountAcc);
+  ws.colmask = reinterpret_cast<unsigned *>(scratch + kOffColmask);
+  ws.arrive_route = reinterpret_cast<int *>(scratch + kOffArrive);
+  ws.mask_words = kStaticMaskWords;
+  // the shared array keeps whatever the last call (possibly an aborted one) left: clear the accumulators
+  if (cudaMemsetAsync(scratch + kOffZero, 0, kZeroBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MOESPEC_ERR_CUDA;
   ws.active = reinterpret_cast<int *>(scratch + kOffActive);
   ws.row2expert = reinterpret_cast<int *>(scratch + kOffRow2Exp);
   ws.stats = reinterpret_cast<moespec_stats *>(scratch + kOffStats);

@@ -5,11 +5,16 @@
 // per-expert gather order (Appendix C).
 //
 // Two launches:
-//   router_topk_kernel   one warp per (token, expert) dot product; the CTA that
-//                        finishes a token's last logit also runs that token's
-//                        softmax and top-k (a counter, never a wait)
-//   route_kernel         one CTA: scores, shortlist, re-routing, scan, gather
-//                        order, work-unit list, statistics
+//   router_topk_kernel   router dot products; the CTA that finishes a token
+//                        tile's last logit also runs those tokens' softmax and
+//                        top-k and adds their probabilities to the per-expert
+//                        scores (a counter, never a wait)
+//   route_kernel         eight tokens per CTA: every CTA ranks the scores itself
+//                        (shortlist), re-routes its tokens, and the CTA that
+//                        finishes last does the scan, the gather order, the
+//                        work-unit list and the statistics
+// Scores are accumulated as 2^-52 fixed-point integers, so the sum does not
+// depend on the order in which tokens arrive and identical experts tie exactly.
 // A stand-alone softmax/top-k kernel serves callers that inject logits.
 #include "internal.h"
 #include <math_constants.h>
@@ -56,9 +61,11 @@ __device__ __forceinline__ int warp_take_best(const uint32_t (&key)[W], uint32_t
 }
 
 // Softmax (Eq. 1, fp64) and natural top-k (Eq. 2) of one token by one warp.
+constexpr double kScoreScale = 4503599627370496.0;   // 2^52
+
 template <int W>
 __device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int k, double *prob_row, int *topk_row,
-                                                   int lane) {
+                                                   unsigned long long *score_fx, int *natcnt, int lane) {
   float v[W];
   uint32_t key[W];
   uint32_t valid = 0;
@@ -87,16 +94,24 @@ __device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(kFull, sum, o);
 #pragma unroll
   for (int s = 0; s < W; ++s)
-    if ((valid >> s) & 1u) prob_row[lane + 32 * s] = e[s] / sum;
+    if ((valid >> s) & 1u) {
+      const double p = e[s] / sum;
+      prob_row[lane + 32 * s] = p;
+      atomicAdd(score_fx + lane + 32 * s, (unsigned long long)__double2ull_rn(p * kScoreScale));   // Eq. 5
+    }
   const int mine = warp_take_best<W>(key, valid, k, lane);
-  if (lane < k) topk_row[lane] = mine;
+  if (lane < k) {
+    topk_row[lane] = mine;
+    if (mine >= 0) atomicAdd(natcnt + mine, 1);
+  }
 }
 
-__device__ __forceinline__ void token_phase(const float *zrow, int N, int k, double *prob_row, int *topk_row, int lane) {
-  if (N <= 32) token_softmax_topk<1>(zrow, N, k, prob_row, topk_row, lane);
-  else if (N <= 64) token_softmax_topk<2>(zrow, N, k, prob_row, topk_row, lane);
-  else if (N <= 128) token_softmax_topk<4>(zrow, N, k, prob_row, topk_row, lane);
-  else token_softmax_topk<8>(zrow, N, k, prob_row, topk_row, lane);
+__device__ __forceinline__ void token_phase(const float *zrow, int N, int k, double *prob_row, int *topk_row,
+                                            unsigned long long *score_fx, int *natcnt, int lane) {
+  if (N <= 32) token_softmax_topk<1>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
+  else if (N <= 64) token_softmax_topk<2>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
+  else if (N <= 128) token_softmax_topk<4>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
+  else token_softmax_topk<8>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
 }
 
 // ---------------------------------------------------------------------------
@@ -111,8 +126,8 @@ __device__ __forceinline__ void token_phase(const float *zrow, int N, int k, dou
 template <typename T, int TT>
 __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                           const float *__restrict__ bias, float *logits,
-                                                          double *prob, int *topk_idx, int *arrive, int M, int N,
-                                                          int d, int k) {
+                                                          double *prob, int *topk_idx, unsigned long long *score_fx,
+                                                          int *natcnt, int *arrive, int M, int N, int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.y * TT;
   const int i = blockIdx.x * 8 + warp;
@@ -172,7 +187,7 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   __syncthreads();
   if (s_last && warp < TT && t0 + warp < M) {
     const int t = t0 + warp;
-    token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, lane);
+    token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane);
   }
 }
 
@@ -184,10 +199,10 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   if (c.M <= 64)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.arrive, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
   return launch_kernel(router_topk_kernel<T, 8>, dim3(ex_tiles, (c.M + 7) / 8), dim3(256), 0, c.stream,
                        (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                       ws.arrive, c.M, D.n_experts, D.d, c.k);
+                       ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
@@ -195,12 +210,15 @@ cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
 }
 
 // Softmax and top-k from caller-supplied logits: one warp per token.
-__global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, double *prob, int *topk_idx, int M,
-                                                           int N, int k) {
+__global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, double *prob, int *topk_idx,
+                                                           unsigned long long *score_fx, int *natcnt, int M, int N,
+                                                           int k) {
   const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
   pdl_trigger();
   pdl_wait();
-  if (t < M) token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, threadIdx.x & 31);
+  if (t < M)
+    token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt,
+                threadIdx.x & 31);
 }
 
 __device__ __forceinline__ double shfl_double(double x, int src) {
@@ -225,231 +243,233 @@ struct RouteArgs {
   long long expert_bytes;       // 3*d*f*sizeof(dtype)
 };
 
+constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
+
+// Probability of expert `idx` from the row a warp holds in registers (lane l owns experts l, l+32, ...).
+template <int W>
+__device__ __forceinline__ double row_value(const double (&p)[W], int idx) {
+  const int slot = idx >> 5;
+  double mine = 0.0;
+#pragma unroll
+  for (int s = 0; s < W; ++s) {
+    const double v = shfl_double(p[s], idx & 31);   // every lane names its own source lane
+    if (s == slot) mine = v;
+  }
+  return mine;
+}
+
 // Re-routing of one token (Eq. 7 / Eq. 8) with its mixing weights (Section 3.3); lane r owns slot r.
+// key[] / p[] are the token's logit keys and probabilities, valid says which slots exist.
 template <int W>
 __device__ __forceinline__ void token_reroute(const RouteArgs &a, int t, int nS, const uint32_t *s_Smask,
-                                              uint32_t *colmask, int mw, int lane) {
+                                              const uint32_t (&key)[W], const double (&p)[W], int nat, int lane) {
   const Workspace &ws = a.ws;
-  const int N = a.N, k = a.k;
+  const int k = a.k;
+  const bool nat_kept = nat >= 0 && ((s_Smask[nat >> 5] >> (nat & 31)) & 1u);
   int mine = -1;        // kept expert of slot `lane`
   int base = -1;        // expert whose probability enters the renormalisation sum at position `lane`
   if (a.policy == MOESPEC_SUBSTITUTION) {
-    uint32_t key[W];
-    uint32_t valid = 0;
+    // The surviving natural experts outrank every other member of S (they are the global top-k), so
+    // top-k within S = survivors in their order, then the best of S \ T_k for the slots that are left.
+    const uint32_t surv = __ballot_sync(kFull, nat_kept);
+    const int n_surv = __popc(surv);
+    const int want = min(k, nS);
+    const unsigned src = __fns(surv, 0, lane + 1);            // lane of the (lane+1)-th survivor
+    const int from_nat = __shfl_sync(kFull, nat, src < 32u ? (int)src : 0);
+    if (lane < n_surv) mine = from_nat;
+    if (n_surv < want) {
+      // candidates: members of S that are not in the natural top-k
+      uint32_t valid = 0;
 #pragma unroll
-    for (int s = 0; s < W; ++s) {
-      const int idx = lane + 32 * s;
-      key[s] = 0;
-      if (idx < N && ((s_Smask[s] >> lane) & 1u)) {
-        key[s] = order_key(a.logits[(size_t)t * N + idx]);
-        valid |= 1u << s;
+      for (int s = 0; s < W; ++s)
+        if ((s_Smask[s] >> lane) & 1u) valid |= 1u << s;
+      for (int r = 0; r < k; ++r) {
+        const int e = __shfl_sync(kFull, nat, r);
+        if (e >= 0 && (e & 31) == lane) valid &= ~(1u << (e >> 5));
       }
+      const int sub = warp_take_best<W>(key, valid, want - n_surv, lane);
+      const int shifted = __shfl_sync(kFull, sub, (lane - n_surv) & 31);
+      if (lane >= n_surv && lane < want) mine = shifted;
     }
-    mine = warp_take_best<W>(key, valid, min(k, nS), lane);
     base = mine;                                   // weights over the constrained selection
-  } else if (lane < k) {
-    const int idx = ws.topk_idx[(size_t)t * k + lane];
-    const bool keep = idx >= 0 && ((s_Smask[idx >> 5] >> (idx & 31)) & 1u);
-    mine = keep ? idx : -1;
-    base = idx;                                    // weights over the original top-k set
+  } else {
+    mine = nat_kept ? nat : -1;
+    base = nat;                                    // weights over the original top-k set
   }
-  const double p_mine = mine >= 0 ? ws.prob[(size_t)t * N + mine] : 0.0;
-  const double p_base = base >= 0 ? (base == mine ? p_mine : ws.prob[(size_t)t * N + base]) : 0.0;
+  const double p_mine = row_value<W>(p, mine >= 0 ? mine : 0);
+  double p_base = p_mine;
+  if (a.policy != MOESPEC_SUBSTITUTION) p_base = row_value<W>(p, base >= 0 ? base : 0);   // warp-uniform branch
   double denom = 1.0;
   if (a.renormalize) {
-    denom = 0.0;
-    for (int r = 0; r < k; ++r) denom += shfl_double(p_base, r);   // rank order
+    denom = (lane < k && base >= 0) ? p_base : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) denom += shfl_xor_double(denom, o);
   }
   if (lane < k) {
     ws.assign_idx[(size_t)t * k + lane] = mine;
     ws.gate_w[(size_t)t * k + lane] = mine >= 0 ? (float)(p_mine / denom) : 0.f;
-    if (mine >= 0) atomicOr(&colmask[(size_t)mine * mw + (t >> 5)], 1u << (t & 31));
+    if (mine >= 0) {
+      atomicAdd(ws.count_acc + mine, 1);
+      atomicOr(ws.colmask + (size_t)mine * ws.mask_words + (t >> 5), 1u << (t & 31));
+    }
   }
 }
 
+template <int W>
+__device__ __forceinline__ void route_token(const RouteArgs &a, int t, int nS, const uint32_t *s_Smask,
+                                            const uint32_t (&key)[W], const double (&p)[W], int nat, int lane) {
+  token_reroute<W>(a, t, nS, s_Smask, key, p, nat, lane);
+}
+
 // ---------------------------------------------------------------------------
-// K2: everything between the per-token top-k and the expert FFNs, in one CTA.
-// The data is tiny (M*N <= a few 10k values); one CTA keeps every ranking
-// deterministic and needs no inter-CTA synchronisation.  Dynamic shared memory:
-//   part[nwarps][N]  fp64 partial scores (warp w adds its tokens w, w+32, ... in
-//                    ascending order; the partials are combined in a fixed tree)
-//   colmask[N][mw]   bit t of row i: expert i is in A(t)
+// K2: shortlist, re-routing and gather order.  Grid ceil(M/8), 256 threads: one
+// warp per token.  Every CTA ranks the N scores itself (rank by counting under
+// (score descending, index ascending)), which costs less than a grid-wide
+// exchange.  Tokens add their kept experts to global counters and bit masks;
+// the CTA that arrives last turns them into offsets, rows and work units and
+// clears the accumulators for the next call.
 // ---------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
-  extern __shared__ __align__(16) unsigned char route_smem[];
-  __shared__ double s_score[kMaxExperts];
+template <int W>
+__global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
+  __shared__ unsigned long long s_score[kMaxExperts];
   __shared__ int s_cand[kMaxExperts];
-  __shared__ int s_natcnt[kMaxExperts];
   __shared__ int s_count[kMaxExperts];
   __shared__ int s_offset[kMaxExperts + 1];
   __shared__ int s_unit_base[kMaxExperts + 1];
   __shared__ int s_Srank[kMaxExperts];
   __shared__ uint32_t s_Smask[kMaskWords];
-  __shared__ unsigned long long s_warp_tot[8];
-  __shared__ int s_nS, s_nactive;
+  __shared__ unsigned long long s_warp_tot[kRouteWarps];
+  __shared__ int s_nactive, s_last;
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = a.M, N = a.N, k = a.k;
-  const int mw = (M + 31) >> 5;
+  const int mw = a.ws.mask_words;
   const Workspace &ws = a.ws;
-  double *s_part = reinterpret_cast<double *>(route_smem);
-  uint32_t *colmask = reinterpret_cast<uint32_t *>(route_smem + (size_t)nwarps * N * sizeof(double));
+  const int t = blockIdx.x * kRouteWarps + warp;
 
-#ifdef MOESPEC_ROUTE_TIMING
-  long long tmark[8];
-  int nmark = 0;
-#define ROUTE_MARK() do { if (tid == 0) tmark[nmark++] = clock64(); } while (0)
-#else
-#define ROUTE_MARK() do { } while (0)
-#endif
   pdl_trigger();
   pdl_wait();
-#ifdef MOESPEC_ROUTE_TIMING
-  for (int rep = 0; rep < 2; ++rep) {
-  nmark = 0;
-  __syncthreads();
-#endif
-  ROUTE_MARK();
+
+  // ---- this warp's token: logit keys, probabilities, natural top-k (all loads issued up front)
+  uint32_t key[W];
+  double p[W];
+  int nat = -1;
+#pragma unroll
+  for (int s = 0; s < W; ++s) {
+    const int idx = lane + 32 * s;
+    key[s] = 0;
+    p[s] = 0.0;
+    if (t < M && idx < N) {
+      key[s] = order_key(a.logits[(size_t)t * N + idx]);
+      p[s] = ws.prob[(size_t)t * N + idx];
+    }
+  }
+  if (t < M && lane < k) nat = ws.topk_idx[(size_t)t * k + lane];
+
+  // ---- scores (Eq. 5), union (Eq. 3), top-B shortlist
   if (tid < kMaskWords) s_Smask[tid] = 0;
-  if (tid == 0) *ws.status = 0;
-  for (int i = tid; i < N; i += blockDim.x) s_natcnt[i] = 0;
-  for (int i = tid; i < N * mw; i += blockDim.x) colmask[i] = 0;
-  __syncthreads();
-
-  // ---- phase A: natural counts (Eq. 3) and partial scores (Eq. 5)
-  for (int item = tid; item < M * k; item += blockDim.x) {
-    const int e = ws.topk_idx[item];
-    if (e >= 0) atomicAdd(&s_natcnt[e], 1);
-  }
-  {
-    double part[kMaskWords];
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s) part[s] = 0.0;
-    for (int t = warp; t < M; t += nwarps) {
-#pragma unroll
-      for (int s = 0; s < kMaskWords; ++s)
-        if (lane + 32 * s < N) part[s] += ws.prob[(size_t)t * N + lane + 32 * s];
-    }
-#pragma unroll
-    for (int s = 0; s < kMaskWords; ++s)
-      if (lane + 32 * s < N) s_part[(size_t)warp * N + lane + 32 * s] = part[s];
+  for (int i = tid; i < N; i += blockDim.x) {
+    s_score[i] = __ldcg(ws.score_fx + i);
+    s_cand[i] = (a.shortlist == MOESPEC_FROM_UNION) ? (__ldcg(ws.natcnt_acc + i) > 0) : 1;
   }
   __syncthreads();
-  ROUTE_MARK();
-
-  // ---- phase B: scores (Eq. 5), union (Eq. 3), top-B shortlist by counting under (score desc, index asc)
-  for (int i = warp; i < N; i += nwarps) {
-    double s = lane < nwarps ? s_part[(size_t)lane * N + i] : 0.0;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += shfl_xor_double(s, o);
-    if (lane == 0) {
-      s_score[i] = s;
-      ws.score[i] = s;
-      s_cand[i] = (a.shortlist == MOESPEC_FROM_UNION) ? (s_natcnt[i] > 0) : 1;
-    }
-  }
-  __syncthreads();
-  const int n_union = __syncthreads_count(tid < N && s_natcnt[tid] > 0);
-  const int n_cand = __syncthreads_count(tid < N && s_cand[tid]);
+  int n_cand = 0;
+  for (int i = lane; i < N; i += 32) n_cand += s_cand[i];
+  n_cand = __reduce_add_sync(kFull, n_cand);
   const int nS = min(a.B, n_cand);
-  for (int i = warp; i < N; i += nwarps) {
+  for (int i = warp; i < N; i += kRouteWarps) {
     if (!s_cand[i]) continue;
-    const double si = s_score[i];
+    const unsigned long long si = s_score[i];
     int ahead = 0;
     for (int j = lane; j < N; j += 32)
       if (s_cand[j]) {
-        const double sj = s_score[j];
+        const unsigned long long sj = s_score[j];
         ahead += (sj > si || (sj == si && j < i)) ? 1 : 0;
       }
     const int rank = __reduce_add_sync(kFull, ahead);
     if (lane == 0 && rank < nS) {
-      ws.S_rank[rank] = i;
       s_Srank[rank] = i;
       atomicOr(&s_Smask[i >> 5], 1u << (i & 31));
+      if (blockIdx.x == 0) ws.S_rank[rank] = i;
     }
   }
-  if (tid == 0) s_nS = nS;
   __syncthreads();
-  ROUTE_MARK();
 
-  // ---- phase C: re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3), one warp per token
-  for (int t = warp; t < M; t += nwarps) {
-    if (N <= 32) token_reroute<1>(a, t, nS, s_Smask, colmask, mw, lane);
-    else if (N <= 64) token_reroute<2>(a, t, nS, s_Smask, colmask, mw, lane);
-    else if (N <= 128) token_reroute<4>(a, t, nS, s_Smask, colmask, mw, lane);
-    else token_reroute<8>(a, t, nS, s_Smask, colmask, mw, lane);
+  // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
+  if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
+
+  // ---- the CTA that arrives last finishes the call
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int prev = atomicAdd(ws.arrive_route, 1);
+    s_last = (prev == (int)gridDim.x - 1);
+    if (s_last) __threadfence();
   }
   __syncthreads();
-  ROUTE_MARK();
+  if (!s_last) return;
 
-  // ---- phase D: rows per expert and exclusive scans of rows, token chunks and active experts
+  // rows per expert and exclusive scans of rows, token chunks and active experts (Appendix C gather)
   {
-    int c = 0;
-    if (tid < N)
-      for (int w = 0; w < mw; ++w) c += __popc(colmask[(size_t)tid * mw + w]);
+    const int c = tid < N ? __ldcg(ws.count_acc + tid) : 0;
     const int chunks = (c + kMaxTokChunk - 1) / kMaxTokChunk;
     // rows in bits 0..23, chunks in bits 24..43, active flag in bits 44..
-    unsigned long long v = (unsigned long long)c | ((unsigned long long)chunks << 24) |
-                           ((unsigned long long)(c > 0) << 44);
+    const unsigned long long v = (unsigned long long)c | ((unsigned long long)chunks << 24) |
+                                 ((unsigned long long)(c > 0) << 44);
     unsigned long long inc = v;
-    if (tid < kMaxExperts) {
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned long long up = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += up;
-      }
-      if (lane == 31) s_warp_tot[warp] = inc;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long up = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += up;
     }
+    if (lane == 31) s_warp_tot[warp] = inc;
     __syncthreads();
-    if (tid < kMaxExperts) {
-      unsigned long long pre = inc - v;
-      for (int w = 0; w < warp; ++w) pre += s_warp_tot[w];
-      if (tid < N) {
-        const int row0 = (int)(pre & 0xFFFFFFull), ub = (int)((pre >> 24) & 0xFFFFFull), ai = (int)(pre >> 44);
-        s_count[tid] = c;
-        s_offset[tid] = row0;
-        s_unit_base[tid] = ub;
-        ws.count[tid] = c;
-        ws.offset[tid] = row0;
-        if (c > 0) ws.active[ai] = tid;
-        if (tid == N - 1) {
-          s_offset[N] = row0 + c;
-          ws.offset[N] = row0 + c;
-          s_unit_base[N] = ub + chunks;
-          s_nactive = ai + (c > 0);
-        }
+    unsigned long long pre = inc - v;
+    for (int w = 0; w < warp; ++w) pre += s_warp_tot[w];
+    if (tid < N) {
+      const int row0 = (int)(pre & 0xFFFFFFull), ub = (int)((pre >> 24) & 0xFFFFFull), ai = (int)(pre >> 44);
+      s_count[tid] = c;
+      s_offset[tid] = row0;
+      s_unit_base[tid] = ub;
+      ws.count[tid] = c;
+      ws.offset[tid] = row0;
+      ws.score[tid] = (double)s_score[tid] * (1.0 / kScoreScale);
+      if (c > 0) ws.active[ai] = tid;
+      if (tid == N - 1) {
+        s_offset[N] = row0 + c;
+        ws.offset[N] = row0 + c;
+        s_unit_base[N] = ub + chunks;
+        s_nactive = ai + (c > 0);
       }
     }
   }
   __syncthreads();
-  ROUTE_MARK();
 
-  // ---- phase E: rows ordered by (expert ascending, token ascending): the row of (t, e) is
-  //      offset[e] + number of tokens below t that were also routed to e
+  // rows ordered by (expert ascending, token ascending): the row of (t, e) is
+  // offset[e] + number of tokens below t that were also routed to e
   for (int item = tid; item < M * k; item += blockDim.x) {
-    const int t = item / k;
-    const int e = ws.assign_idx[item];
+    const int tt = item / k;
+    const int e = __ldcg(ws.assign_idx + item);
     int row = -1;
     if (e >= 0) {
-      const uint32_t *cm = colmask + (size_t)e * mw;
-      int below = __popc(cm[t >> 5] & ((1u << (t & 31)) - 1u));
-      for (int w = 0; w < (t >> 5); ++w) below += __popc(cm[w]);
+      const unsigned *cm = ws.colmask + (size_t)e * mw;
+      int below = __popc(__ldcg(cm + (tt >> 5)) & ((1u << (tt & 31)) - 1u));
+      for (int w = 0; w < (tt >> 5); ++w) below += __popc(__ldcg(cm + w));
       row = s_offset[e] + below;
-      ws.perm_row2tok[row] = t;
+      ws.perm_row2tok[row] = tt;
       ws.row2expert[row] = e;
     }
     ws.tokslot2row[item] = row;
   }
-  ROUTE_MARK();
 
-  // ---- phase F: tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all
-  //      down units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
+  // tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all down
+  // units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
   const int n_chunks = s_unit_base[N];
   if (a.tiles_up > 0) {
     const int n_up = n_chunks * a.tiles_up;
     for (int i = tid; i < n_chunks; i += blockDim.x) ws.ready[i] = 0;
     if (tid == 0) *ws.unit_counter = 0;
-    for (int i = warp; i < N; i += nwarps) {
+    for (int i = warp; i < N; i += kRouteWarps) {
       const int cnt = s_count[i];
       if (cnt == 0) continue;
       const int chunks = (cnt + kMaxTokChunk - 1) / kMaxTokChunk;
@@ -465,18 +485,20 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
     }
   }
 
+  // statistics, then clear the accumulators for the next call
+  const int n_union = __syncthreads_count(tid < N && __ldcg(ws.natcnt_acc + tid) > 0);
   if (tid == 0) {
     const int R = s_offset[N];
-    ws.counters[0] = s_nS;
+    ws.counters[0] = nS;
     ws.counters[1] = s_nactive;
     ws.counters[2] = R;
     ws.counters[3] = n_chunks * a.tiles_up;
     ws.counters[4] = n_chunks * a.tiles_down;
     double cov = 0.0;
-    for (int r = 0; r < s_nS; ++r) cov += s_score[s_Srank[r]];
+    for (int r = 0; r < nS; ++r) cov += (double)s_score[s_Srank[r]] * (1.0 / kScoreScale);
     moespec_stats st;
     st.n_union = n_union;
-    st.n_shortlist = s_nS;
+    st.n_shortlist = nS;
     st.n_active = s_nactive;
     st.n_rows = R;
     st.n_dropped = M * k - R;
@@ -484,17 +506,17 @@ __global__ void __launch_bounds__(1024) route_kernel(RouteArgs a) {
     st.coverage = M > 0 ? cov / (double)M : 0.0;
     st.weight_bytes = (long long)s_nactive * a.expert_bytes;
     *ws.stats = st;
-#ifdef MOESPEC_ROUTE_TIMING
-    tmark[nmark++] = clock64();
-    printf("route phases (cycles): A %lld B %lld C %lld D %lld E %lld F+stats %lld total %lld\n", tmark[1] - tmark[0],
-           tmark[2] - tmark[1], tmark[3] - tmark[2], tmark[4] - tmark[3], tmark[5] - tmark[4], tmark[6] - tmark[5],
-           tmark[6] - tmark[0]);
-#endif
+    *ws.status = 0;
+    *ws.arrive_route = 0;
   }
-#ifdef MOESPEC_ROUTE_TIMING
   __syncthreads();
+  for (int i = tid; i < N; i += blockDim.x) {
+    ws.score_fx[i] = 0ull;
+    ws.natcnt_acc[i] = 0;
+    ws.count_acc[i] = 0;
   }
-#endif
+  const int used_words = (M + 31) >> 5;
+  for (int i = tid; i < N * used_words; i += blockDim.x) ws.colmask[(size_t)(i / used_words) * mw + (i % used_words)] = 0u;
 }
 
 static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) {
@@ -508,22 +530,20 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.tiles_up = tc ? D.f / kTile : 0;
   a.tiles_down = tc ? D.d / kTile : 0;
   a.expert_bytes = 3LL * D.d * D.f * (D.dtype == MOESPEC_BF16 ? 2 : 4);
-  const int threads = 1024;
-  const size_t smem = (size_t)(threads / 32) * a.N * sizeof(double) + (size_t)a.N * ((c.M + 31) / 32) * sizeof(uint32_t);
-  if (smem > 40 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(route_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-  }
-  return launch_kernel(route_kernel, dim3(1), dim3(threads), smem, c.stream, a);
+  const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
+  if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
+  if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);
+  if (a.N <= 128) return launch_kernel(route_kernel<4>, grid, block, 0, c.stream, a);
+  return launch_kernel(route_kernel<8>, grid, block, 0, c.stream, a);
 }
 
-// Routing after router_topk_kernel has filled logits, prob and topk_idx.
+// Routing after router_topk_kernel has filled logits, prob, topk_idx and the score accumulators.
 cudaError_t launch_route_after_router(const LaunchCtx &c) { return launch_route_kernel(c, c.ws->logits); }
 
 // Routing from caller-supplied logits: per-token softmax/top-k first (two launches).
 cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
   cudaError_t e = launch_kernel(softmax_topk_kernel, dim3((c.M + 3) / 4), dim3(128), 0, c.stream, logits, c.ws->prob,
-                                c.ws->topk_idx, c.M, c.desc->n_experts, c.k);
+                                c.ws->topk_idx, c.ws->score_fx, c.ws->natcnt_acc, c.M, c.desc->n_experts, c.k);
   if (e != cudaSuccess) return e;
   return launch_route_kernel(c, logits);
 }
