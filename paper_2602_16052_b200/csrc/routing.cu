@@ -26,6 +26,7 @@ __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 
 constexpr unsigned kFull = 0xffffffffu;
+constexpr double kScoreScale = 4503599627370496.0;   // 2^52: scores are sums of round(p * 2^52)
 constexpr int kNone = 0x7fffffff;
 
 // Monotone map float -> uint32 (larger float, larger key); -0 and +0 share a key.
@@ -60,24 +61,19 @@ __device__ __forceinline__ int warp_take_best(const uint32_t (&key)[W], uint32_t
   return mine;
 }
 
-// Softmax (Eq. 1, fp64) and natural top-k (Eq. 2) of one token by one warp.
-constexpr double kScoreScale = 4503599627370496.0;   // 2^52
-
+// Softmax of one token by one warp (Eq. 1, fp64); adds the probabilities to the per-expert scores (Eq. 5).
 template <int W>
-__device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int k, double *prob_row, int *topk_row,
-                                                   unsigned long long *score_fx, int *natcnt, int lane) {
+__device__ __forceinline__ void token_softmax(const float *zrow, int N, double *prob_row, unsigned long long *score_fx,
+                                              int lane) {
   float v[W];
-  uint32_t key[W];
   uint32_t valid = 0;
   float mx = -CUDART_INF_F;
 #pragma unroll
   for (int s = 0; s < W; ++s) {
     const int idx = lane + 32 * s;
     v[s] = -CUDART_INF_F;
-    key[s] = 0;
     if (idx < N) {
       v[s] = __ldcg(zrow + idx);          // written by other CTAs of this launch: read through L2
-      key[s] = order_key(v[s]);
       valid |= 1u << s;
       mx = fmaxf(mx, v[s]);
     }
@@ -97,8 +93,24 @@ __device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int
     if ((valid >> s) & 1u) {
       const double p = e[s] / sum;
       prob_row[lane + 32 * s] = p;
-      atomicAdd(score_fx + lane + 32 * s, (unsigned long long)__double2ull_rn(p * kScoreScale));   // Eq. 5
+      atomicAdd(score_fx + lane + 32 * s, (unsigned long long)__double2ull_rn(p * kScoreScale));
     }
+}
+
+// Natural top-k of one token by one warp (Eq. 2); counts the token towards its experts (Eq. 3).
+template <int W>
+__device__ __forceinline__ void token_topk(const float *zrow, int N, int k, int *topk_row, int *natcnt, int lane) {
+  uint32_t key[W];
+  uint32_t valid = 0;
+#pragma unroll
+  for (int s = 0; s < W; ++s) {
+    const int idx = lane + 32 * s;
+    key[s] = 0;
+    if (idx < N) {
+      key[s] = order_key(__ldcg(zrow + idx));
+      valid |= 1u << s;
+    }
+  }
   const int mine = warp_take_best<W>(key, valid, k, lane);
   if (lane < k) {
     topk_row[lane] = mine;
@@ -106,12 +118,22 @@ __device__ __forceinline__ void token_softmax_topk(const float *zrow, int N, int
   }
 }
 
+// which: bit 0 = softmax, bit 1 = top-k
 __device__ __forceinline__ void token_phase(const float *zrow, int N, int k, double *prob_row, int *topk_row,
-                                            unsigned long long *score_fx, int *natcnt, int lane) {
-  if (N <= 32) token_softmax_topk<1>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
-  else if (N <= 64) token_softmax_topk<2>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
-  else if (N <= 128) token_softmax_topk<4>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
-  else token_softmax_topk<8>(zrow, N, k, prob_row, topk_row, score_fx, natcnt, lane);
+                                            unsigned long long *score_fx, int *natcnt, int lane, int which = 3) {
+  if (N <= 32) {
+    if (which & 1) token_softmax<1>(zrow, N, prob_row, score_fx, lane);
+    if (which & 2) token_topk<1>(zrow, N, k, topk_row, natcnt, lane);
+  } else if (N <= 64) {
+    if (which & 1) token_softmax<2>(zrow, N, prob_row, score_fx, lane);
+    if (which & 2) token_topk<2>(zrow, N, k, topk_row, natcnt, lane);
+  } else if (N <= 128) {
+    if (which & 1) token_softmax<4>(zrow, N, prob_row, score_fx, lane);
+    if (which & 2) token_topk<4>(zrow, N, k, topk_row, natcnt, lane);
+  } else {
+    if (which & 1) token_softmax<8>(zrow, N, prob_row, score_fx, lane);
+    if (which & 2) token_topk<8>(zrow, N, k, topk_row, natcnt, lane);
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -134,6 +156,9 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   __shared__ int s_last;
   pdl_trigger();
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+#ifdef MOESPEC_ROUTE_TIMING
+  const long long tm0 = clock64();
+#endif
   if (i < N) {
     constexpr int VEC = 16 / sizeof(T);
     constexpr int U = 8;
@@ -146,21 +171,28 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
 #pragma unroll
       for (int u = 0; u < U; ++u)
         if (j0 + u * 32 * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(w + j0 + u * 32 * VEC);
+      // two tokens per pass: their loads are all issued before the first FMA
 #pragma unroll
-      for (int tt = 0; tt < TT; ++tt) {
-        if (t0 + tt >= M) break;
-        const T *h = hidden + (size_t)(t0 + tt) * d;
-        uint4 rh[U];
+      for (int tt = 0; tt < TT; tt += 2) {
+        uint4 rh[2][U];
 #pragma unroll
-        for (int u = 0; u < U; ++u)
-          if (j0 + u * 32 * VEC < d) rh[u] = *reinterpret_cast<const uint4 *>(h + j0 + u * 32 * VEC);
+        for (int q = 0; q < 2; ++q) {
+          const int tq = min(t0 + tt + q, M - 1);           // clamp: out-of-range tokens repeat the last row
+          const T *h = hidden + (size_t)tq * d;
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          if (j0 + u * 32 * VEC < d) {
-            const T *ew = reinterpret_cast<const T *>(&rw[u]);
-            const T *eh = reinterpret_cast<const T *>(&rh[u]);
+          for (int u = 0; u < U; ++u)
+            if (j0 + u * 32 * VEC < d) rh[q][u] = *reinterpret_cast<const uint4 *>(h + j0 + u * 32 * VEC);
+        }
 #pragma unroll
-            for (int v = 0; v < VEC; ++v) acc[tt] = fmaf(to_float(ew[v]), to_float(eh[v]), acc[tt]);
+        for (int q = 0; q < 2; ++q) {
+#pragma unroll
+          for (int u = 0; u < U; ++u) {
+            if (j0 + u * 32 * VEC < d) {
+              const T *ew = reinterpret_cast<const T *>(&rw[u]);
+              const T *eh = reinterpret_cast<const T *>(&rh[q][u]);
+#pragma unroll
+              for (int v = 0; v < VEC; ++v) acc[tt + q] = fmaf(to_float(ew[v]), to_float(eh[v]), acc[tt + q]);
+            }
           }
         }
       }
@@ -176,6 +208,9 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
     if (lane == 0) __threadfence();
   }
   __syncthreads();
+#ifdef MOESPEC_ROUTE_TIMING
+  const long long tm1 = clock64();
+#endif
   if (threadIdx.x == 0) {
     const int prev = atomicAdd(&arrive[blockIdx.y], 1);
     s_last = (prev == (int)gridDim.x - 1);
@@ -185,10 +220,23 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
     }
   }
   __syncthreads();
-  if (s_last && warp < TT && t0 + warp < M) {
-    const int t = t0 + warp;
-    token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane);
+#ifdef MOESPEC_ROUTE_TIMING
+  const long long tm2 = clock64();
+#endif
+  if (s_last) {
+    // softmax and top-k are independent chains: with up to four tokens they run on different warps
+    const bool split = 2 * TT <= 8;
+    const int tt = split ? (warp % TT) : warp;
+    const int which = split ? (warp < TT ? 1 : 2) : 3;
+    const int t = t0 + tt;
+    if (tt < TT && (split ? warp < 2 * TT : true) && t < M)
+      token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane,
+                  which);
   }
+#ifdef MOESPEC_ROUTE_TIMING
+  if (s_last && threadIdx.x == 0 && blockIdx.y == 0)
+    printf("router (cycles): dot %lld arrive %lld token %lld\n", tm1 - tm0, tm2 - tm1, clock64() - tm2);
+#endif
 }
 
 template <typename T>
@@ -197,6 +245,10 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   const Workspace &ws = *c.ws;
   const int ex_tiles = (D.n_experts + 7) / 8;
   if (c.M <= 64)
+    return launch_kernel(router_topk_kernel<T, 2>, dim3(ex_tiles, (c.M + 1) / 2), dim3(256), 0, c.stream,
+                         (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
+  if (c.M <= 128)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
                          ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
@@ -244,6 +296,7 @@ struct RouteArgs {
 };
 
 constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
+constexpr int kColmaskCache = 2048; // words of the expert x token bit matrix the last CTA keeps in shared memory
 
 // Probability of expert `idx` from the row a warp holds in registers (lane l owns experts l, l+32, ...).
 template <int W>
@@ -310,7 +363,7 @@ __device__ __forceinline__ void token_reroute(const RouteArgs &a, int t, int nS,
     ws.gate_w[(size_t)t * k + lane] = mine >= 0 ? (float)(p_mine / denom) : 0.f;
     if (mine >= 0) {
       atomicAdd(ws.count_acc + mine, 1);
-      atomicOr(ws.colmask + (size_t)mine * ws.mask_words + (t >> 5), 1u << (t & 31));
+      atomicOr(ws.colmask + (size_t)mine * ((a.M + 31) >> 5) + (t >> 5), 1u << (t & 31));
     }
   }
 }
@@ -331,7 +384,9 @@ __device__ __forceinline__ void route_token(const RouteArgs &a, int t, int nS, c
 // ---------------------------------------------------------------------------
 template <int W>
 __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
-  __shared__ unsigned long long s_score[kMaxExperts];
+  __shared__ unsigned long long s_score[kMaxExperts];     // ranking key (score + 1, or 0 for a non-candidate)
+  __shared__ unsigned long long s_fx[kMaxExperts];        // fixed-point score
+  __shared__ unsigned s_colmask[kColmaskCache];
   __shared__ int s_cand[kMaxExperts];
   __shared__ int s_count[kMaxExperts];
   __shared__ int s_offset[kMaxExperts + 1];
@@ -339,16 +394,25 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   __shared__ int s_Srank[kMaxExperts];
   __shared__ uint32_t s_Smask[kMaskWords];
   __shared__ unsigned long long s_warp_tot[kRouteWarps];
+  __shared__ int s_chunk_expert[kMaxExperts * 2];     // token chunk -> expert (first 2N chunks; more fall back)
   __shared__ int s_nactive, s_last;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = a.M, N = a.N, k = a.k;
-  const int mw = a.ws.mask_words;
+  const int mw = (a.M + 31) >> 5;     // words per expert row of the bit matrix in this call
   const Workspace &ws = a.ws;
   const int t = blockIdx.x * kRouteWarps + warp;
 
   pdl_trigger();
   pdl_wait();
+#ifdef MOESPEC_ROUTE_TIMING
+  long long tmark[10];
+  int nmark = 0;
+#define ROUTE_MARK() do { if (tid == 0) tmark[nmark++] = clock64(); } while (0)
+#else
+#define ROUTE_MARK() do { } while (0)
+#endif
+  ROUTE_MARK();
 
   // ---- this warp's token: logit keys, probabilities, natural top-k (all loads issued up front)
   uint32_t key[W];
@@ -367,36 +431,46 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   if (t < M && lane < k) nat = ws.topk_idx[(size_t)t * k + lane];
 
   // ---- scores (Eq. 5), union (Eq. 3), top-B shortlist
-  if (tid < kMaskWords) s_Smask[tid] = 0;
-  for (int i = tid; i < N; i += blockDim.x) {
-    s_score[i] = __ldcg(ws.score_fx + i);
-    s_cand[i] = (a.shortlist == MOESPEC_FROM_UNION) ? (__ldcg(ws.natcnt_acc + i) > 0) : 1;
+  int in_union = 0;
+  if (tid < N) {
+    const unsigned long long fx = __ldcg(ws.score_fx + tid);
+    in_union = __ldcg(ws.natcnt_acc + tid) > 0;
+    s_cand[tid] = (a.shortlist == MOESPEC_FROM_UNION) ? in_union : 1;
+    s_score[tid] = s_cand[tid] ? fx + 1ull : 0ull;        // ranking key: candidates first, then by score
+    s_fx[tid] = fx;
   }
-  __syncthreads();
-  int n_cand = 0;
-  for (int i = lane; i < N; i += 32) n_cand += s_cand[i];
-  n_cand = __reduce_add_sync(kFull, n_cand);
+  const int n_union = __syncthreads_count(in_union);
+  ROUTE_MARK();
+  const int n_cand = __syncthreads_count(tid < N && s_cand[tid]);
   const int nS = min(a.B, n_cand);
-  for (int i = warp; i < N; i += kRouteWarps) {
-    if (!s_cand[i]) continue;
-    const unsigned long long si = s_score[i];
-    int ahead = 0;
-    for (int j = lane; j < N; j += 32)
-      if (s_cand[j]) {
+  {
+    // one thread per expert; every thread walks the same j, so the shared-memory reads are broadcasts
+    // Branch-free rank by counting.  s_score holds score+1 for candidates and 0 for the others, so a
+    // non-candidate never outranks a candidate.
+    bool in_S = false;
+    if (tid < N) {
+      const unsigned long long si = s_score[tid];
+      int rank = 0;
+#pragma unroll 16
+      for (int j = 0; j < N; ++j) {
         const unsigned long long sj = s_score[j];
-        ahead += (sj > si || (sj == si && j < i)) ? 1 : 0;
+        rank += (int)((sj > si) | ((sj == si) & (j < tid)));
       }
-    const int rank = __reduce_add_sync(kFull, ahead);
-    if (lane == 0 && rank < nS) {
-      s_Srank[rank] = i;
-      atomicOr(&s_Smask[i >> 5], 1u << (i & 31));
-      if (blockIdx.x == 0) ws.S_rank[rank] = i;
+      in_S = si != 0ull && rank < nS;
+      if (in_S) {
+        s_Srank[rank] = tid;
+        if (blockIdx.x == 0) ws.S_rank[rank] = tid;
+      }
     }
+    const unsigned word = __ballot_sync(kFull, in_S);     // thread index = expert index: warp w owns mask word w
+    if (lane == 0) s_Smask[warp] = word;
   }
   __syncthreads();
+  ROUTE_MARK();
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
+  ROUTE_MARK();
 
   // ---- the CTA that arrives last finishes the call
   __threadfence();
@@ -408,10 +482,15 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   }
   __syncthreads();
   if (!s_last) return;
+  ROUTE_MARK();
 
   // rows per expert and exclusive scans of rows, token chunks and active experts (Appendix C gather)
+  const int used_words = (M + 31) >> 5;
+  const bool cm_cached = N * used_words <= kColmaskCache;
   {
     const int c = tid < N ? __ldcg(ws.count_acc + tid) : 0;
+    if (cm_cached)
+      for (int i = tid; i < N * used_words; i += blockDim.x) s_colmask[i] = __ldcg(ws.colmask + i);
     const int chunks = (c + kMaxTokChunk - 1) / kMaxTokChunk;
     // rows in bits 0..23, chunks in bits 24..43, active flag in bits 44..
     const unsigned long long v = (unsigned long long)c | ((unsigned long long)chunks << 24) |
@@ -433,8 +512,9 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       s_unit_base[tid] = ub;
       ws.count[tid] = c;
       ws.offset[tid] = row0;
-      ws.score[tid] = (double)s_score[tid] * (1.0 / kScoreScale);
+      ws.score[tid] = (double)s_fx[tid] * (1.0 / kScoreScale);
       if (c > 0) ws.active[ai] = tid;
+      for (int cc = 0; cc < chunks && ub + cc < 2 * kMaxExperts; ++cc) s_chunk_expert[ub + cc] = tid;
       if (tid == N - 1) {
         s_offset[N] = row0 + c;
         ws.offset[N] = row0 + c;
@@ -444,58 +524,91 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     }
   }
   __syncthreads();
+  ROUTE_MARK();
 
-  // rows ordered by (expert ascending, token ascending): the row of (t, e) is
-  // offset[e] + number of tokens below t that were also routed to e
-  for (int item = tid; item < M * k; item += blockDim.x) {
-    const int tt = item / k;
-    const int e = __ldcg(ws.assign_idx + item);
-    int row = -1;
-    if (e >= 0) {
-      const unsigned *cm = ws.colmask + (size_t)e * mw;
-      int below = __popc(__ldcg(cm + (tt >> 5)) & ((1u << (tt & 31)) - 1u));
-      for (int w = 0; w < (tt >> 5); ++w) below += __popc(__ldcg(cm + w));
-      row = s_offset[e] + below;
-      ws.perm_row2tok[row] = tt;
-      ws.row2expert[row] = e;
-    }
-    ws.tokslot2row[item] = row;
-  }
-
-  // tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all down
-  // units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
+  // The rest is three independent jobs, each latency-bound, run side by side:
+  //   warps 0-3  row of every (token, slot)       warps 4-6  work-unit list       warp 7  coverage
   const int n_chunks = s_unit_base[N];
-  if (a.tiles_up > 0) {
-    const int n_up = n_chunks * a.tiles_up;
-    for (int i = tid; i < n_chunks; i += blockDim.x) ws.ready[i] = 0;
-    if (tid == 0) *ws.unit_counter = 0;
-    for (int i = warp; i < N; i += kRouteWarps) {
-      const int cnt = s_count[i];
-      if (cnt == 0) continue;
-      const int chunks = (cnt + kMaxTokChunk - 1) / kMaxTokChunk;
-      for (int c = 0; c < chunks; ++c) {
-        const int row0 = s_offset[i] + c * kMaxTokChunk;
-        const int rows = min(kMaxTokChunk, cnt - c * kMaxTokChunk);
-        const int ci = s_unit_base[i] + c;
-        for (int tl = lane; tl < a.tiles_up; tl += 32)
-          ws.units[(size_t)ci * a.tiles_up + tl] = Unit{i, tl, row0, rows, ci, 0, 0, 0};
-        for (int tl = lane; tl < a.tiles_down; tl += 32)
-          ws.units[(size_t)n_up + (size_t)ci * a.tiles_down + tl] = Unit{i, tl, row0, rows, ci, 1, 0, 0};
+  double cov = 0.0;
+  if (warp < 4) {
+    // rows ordered by (expert ascending, token ascending): the row of (t, e) is
+    // offset[e] + number of tokens below t that were also routed to e
+    // thread -> (token, slot) with the slot count padded to a power of two (no integer division)
+    int kshift = 0;
+    while ((1 << kshift) < k) ++kshift;
+    const int slot = tid & ((1 << kshift) - 1);
+    const int tok_step = 128 >> kshift;                    // tokens covered per pass by these 128 threads
+    for (int t0 = tid >> kshift; t0 < M; t0 += 4 * tok_step) {
+      int e[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int tt = t0 + u * tok_step;
+        e[u] = (tt < M && slot < k) ? __ldcg(ws.assign_idx + (size_t)tt * k + slot) : -1;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int tt = t0 + u * tok_step;
+        if (tt >= M || slot >= k) continue;
+        int row = -1;
+        if (e[u] >= 0) {
+          const unsigned *cm = cm_cached ? s_colmask + e[u] * used_words : ws.colmask + (size_t)e[u] * mw;
+          int below = 0;
+          if (cm_cached) {
+            below = __popc(cm[tt >> 5] & ((1u << (tt & 31)) - 1u));
+            for (int w = 0; w < (tt >> 5); ++w) below += __popc(cm[w]);
+          } else {
+            below = __popc(__ldcg(cm + (tt >> 5)) & ((1u << (tt & 31)) - 1u));
+            for (int w = 0; w < (tt >> 5); ++w) below += __popc(__ldcg(cm + w));
+          }
+          row = s_offset[e[u]] + below;
+          ws.perm_row2tok[row] = tt;
+          ws.row2expert[row] = e[u];
+        }
+        ws.tokslot2row[(size_t)tt * k + slot] = row;
       }
     }
+  } else if (warp < 7) {
+    // tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all down
+    // units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
+    if (a.tiles_up > 0) {
+      const int lt = tid - 128, nthr = 96;
+      const int n_up = n_chunks * a.tiles_up, n_down = n_chunks * a.tiles_down;
+      for (int i = lt; i < n_chunks; i += nthr) ws.ready[i] = 0;
+      if (lt == 0) *ws.unit_counter = 0;
+      for (int u = lt; u < n_up + n_down; u += nthr) {
+        const int phase = u >= n_up;
+        const int tiles = phase ? a.tiles_down : a.tiles_up;
+        const int v = phase ? u - n_up : u;
+        const int ci = v / tiles, tl = v - ci * tiles;
+        int e;
+        if (ci < 2 * kMaxExperts) {
+          e = s_chunk_expert[ci];
+        } else {          // more than 2N token chunks (M far beyond 256): search the chunk bases
+          e = 0;
+          while (s_unit_base[e + 1] <= ci) ++e;
+        }
+        const int c = ci - s_unit_base[e];
+        const int row0 = s_offset[e] + c * kMaxTokChunk;
+        const int rows = min(kMaxTokChunk, s_count[e] - c * kMaxTokChunk);
+        ws.units[u] = Unit{e, tl, row0, rows, ci, phase, 0, 0};
+      }
+    }
+  } else {
+    for (int r = lane; r < nS; r += 32) cov += (double)s_fx[s_Srank[r]];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) cov += shfl_xor_double(cov, o);
+    cov *= 1.0 / kScoreScale;
   }
-
-  // statistics, then clear the accumulators for the next call
-  const int n_union = __syncthreads_count(tid < N && __ldcg(ws.natcnt_acc + tid) > 0);
-  if (tid == 0) {
+  ROUTE_MARK();
+  ROUTE_MARK();
+  ROUTE_MARK();
+  if (tid == 224) {         // lane 0 of warp 7, which holds the coverage sum
     const int R = s_offset[N];
     ws.counters[0] = nS;
     ws.counters[1] = s_nactive;
     ws.counters[2] = R;
     ws.counters[3] = n_chunks * a.tiles_up;
     ws.counters[4] = n_chunks * a.tiles_down;
-    double cov = 0.0;
-    for (int r = 0; r < nS; ++r) cov += (double)s_score[s_Srank[r]] * (1.0 / kScoreScale);
     moespec_stats st;
     st.n_union = n_union;
     st.n_shortlist = nS;
@@ -509,14 +622,21 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     *ws.status = 0;
     *ws.arrive_route = 0;
   }
+  if (tid == 0) {
+#ifdef MOESPEC_ROUTE_TIMING
+    tmark[nmark++] = clock64();
+    printf("route (cycles): load+scores %lld shortlist %lld reroute %lld arrive %lld scan %lld rows %lld units %lld stats %lld total %lld\n",
+           tmark[1] - tmark[0], tmark[2] - tmark[1], tmark[3] - tmark[2], tmark[4] - tmark[3], tmark[5] - tmark[4],
+           tmark[6] - tmark[5], tmark[7] - tmark[6], tmark[8] - tmark[7], tmark[8] - tmark[0]);
+#endif
+  }
   __syncthreads();
   for (int i = tid; i < N; i += blockDim.x) {
     ws.score_fx[i] = 0ull;
     ws.natcnt_acc[i] = 0;
     ws.count_acc[i] = 0;
   }
-  const int used_words = (M + 31) >> 5;
-  for (int i = tid; i < N * used_words; i += blockDim.x) ws.colmask[(size_t)(i / used_words) * mw + (i % used_words)] = 0u;
+  for (int i = tid; i < N * used_words; i += blockDim.x) ws.colmask[i] = 0u;
 }
 
 static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) {
