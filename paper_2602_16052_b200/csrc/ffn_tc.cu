@@ -108,11 +108,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// Weights are read once per call: evict-first keeps them from flushing the small hot set (router
+// matrix, gathered rows, h_mid, y) out of L2.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
-                                            int c2) {
+                                            int c2, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
@@ -230,6 +237,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     const int n_up = a.n_units[0], n_total = n_up + a.n_units[1];
     uint32_t it = 0, qi = 0;
     bool ok = true;
+    const uint64_t wpol = l2_evict_first_policy();
     int u = atomicAdd(a.unit_counter, 1);
     while (ok) {
       const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
@@ -265,14 +273,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
         if (un.phase == 0) {
           mbar_expect_tx(full, 2u * kABytes + (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_gate, full, kc * kChunkK, un.tile * kTile, un.expert);
-          tma_load_3d(stage + kABytes, &maps.w_up, full, kc * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage, &maps.w_gate, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
+          tma_load_3d(stage + kABytes, &maps.w_up, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
           for (int b = 0; b < n_pad / kTokBox; ++b)
             tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
         } else if (a.down_double) {
           mbar_expect_tx(full, 2u * kABytes + 2u * (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_down, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert);
-          tma_load_3d(stage + kABytes, &maps.w_down, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage, &maps.w_down, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert, wpol);
+          tma_load_3d(stage + kABytes, &maps.w_down, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert, wpol);
           for (int b = 0; b < n_pad / kTokBox; ++b) {
             tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, (2 * kc) * kChunkK, un.row0 + b * kTokBox);
             tma_load_2d(stage + a.b1_off + b * (kTokBox * 128), map_b, full, (2 * kc + 1) * kChunkK,
@@ -280,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           }
         } else {
           mbar_expect_tx(full, (uint32_t)kABytes + (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_down, full, kc * kChunkK, un.tile * kTile, un.expert);
+          tma_load_3d(stage, &maps.w_down, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
           for (int b = 0; b < n_pad / kTokBox; ++b)
             tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
         }
