@@ -42,9 +42,9 @@ M_TOKENS = 63
 B_HEADLINE = 32
 N_COPIES = 4
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of the two expert-FFN launches of one
-# verify layer (M=63, B=32), from the ncu capture summarised under profiles/; None until captured
-FFN_DRAM_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of the expert-FFN launch of one
+# verify layer (M=63, B=32), from the ncu capture summarised under profiles/
+FFN_DRAM_TRAFFIC_BYTES = 409.6e6   # 404.8 MB read + 4.8 MB written (profiles/ffn_tc_kernel_olmoe_M63_B32.md)
 
 
 def workload_name(cfg):
@@ -190,6 +190,60 @@ def kernel_profile(layers, hiddens, outs, k, B, reps):
     return {name: sum(v) / len(v) for name, v in acc.items()}
 
 
+def run_tables(args, device):
+    """Sweeps over every workload shape (not part of the default run): one JSON line per point."""
+    from paper_2602_16052_b200 import moespec
+    peak, peak_kind = measured_peaks()
+    names = args.tables.split(",")
+    for name in names:
+        cfg = synth.CONFIGS[name]
+        L = cfg.n_layers
+        n_copies = L if L > 1 else (2 if name == "mixtral" else 4)
+        Ms, Bs = synth.SWEEPS[name]["M"], synth.SWEEPS[name]["B"]
+        max_M = max(Ms)
+        weights = [synth.gen_layer(cfg, seed=2000, layer=l, device=device) for l in range(n_copies)]
+        out_dtype = torch.bfloat16 if L > 1 else torch.float32
+        layers = [moespec.Layer(w["router_w"], w["router_bias"], w["w_gate"], w["w_up"], w["w_down"], max_M=max_M,
+                                max_k=cfg.k, policy=moespec.SUBSTITUTION, shortlist=moespec.FROM_ALL, renormalize=True,
+                                residual=L > 1, out_dtype=out_dtype) for w in weights]
+        for M in Ms:
+            x0 = synth.gen_hidden(cfg, M, seed=2000, layer=0, device=device)
+            bufs = [torch.empty_like(x0, dtype=out_dtype) for _ in range(2)]
+            for B in Bs:
+                def one_pass():
+                    if L > 1:        # stack: x <- dtype(x + MoE_l(x)), layer after layer
+                        cur = x0
+                        for l, lay in enumerate(layers):
+                            lay.verify_layer(cur, cfg.k, B, bufs[l % 2])
+                            cur = bufs[l % 2]
+                    else:            # single layer: rotate over independently seeded copies
+                        for lay in layers:
+                            lay.verify_layer(x0, cfg.k, B, bufs[0])
+                reps = max(3, args.steps // len(layers))
+                for _ in range(2):
+                    one_pass()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    one_pass()
+                e1.record()
+                torch.cuda.synchronize()
+                us = e0.elapsed_time(e1) * 1e3 / (reps * len(layers))
+                st = [lay.get_stats() for lay in layers]
+                act = sum(s_["n_active"] for s_ in st) / len(st)
+                uni = sum(s_["n_union"] for s_ in st) / len(st)
+                by = algorithmic_bytes(cfg, M, act, 2 if out_dtype == torch.bfloat16 else 4)
+                print(json.dumps({"table": name, "layers": L, "M": M, "B": B, "us_per_layer": round(us, 2),
+                                  "n_active": round(act, 2), "n_union": round(uni, 2), "MB": round(by / 1e6, 1),
+                                  "GBs": round(by / us / 1e3, 1), "frac_of_" + peak_kind: round(by / us / 1e3 / peak, 3),
+                                  "ideal_us": round(by / peak / 1e3, 1)}), flush=True)
+        for lay in layers:
+            lay.destroy()
+        del layers, weights
+        torch.cuda.empty_cache()
+
+
 def oracle_case(cfg, M, seed):
     L = synth.gen_layer(cfg, seed=seed, layer=0, device="cpu")
     h = synth.gen_hidden(cfg, M, seed=seed, layer=0, device="cpu")
@@ -249,6 +303,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--copies", type=int, default=N_COPIES, help="independently seeded layer copies rotated over")
+    ap.add_argument("--tables", default="", help="comma-separated workload names (tiny is excluded): sweep M and B "
+                    "of each and print one JSON line per point instead of the benchmark line")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed steps (for profiler captures); prints a short line")
     args = ap.parse_args()
@@ -280,6 +336,9 @@ def main():
         t = torch.tensor([x], dtype=torch.float64, device=device)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         return float(t.item())
+
+    if args.tables:
+        return run_tables(args, device)
 
     cfg = synth.CONFIGS[WORKLOAD]
     M, k, B = M_TOKENS, cfg.k, B_HEADLINE

@@ -112,8 +112,10 @@ int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int 
 
 /* Same computation with HOST buffers: copies hidden (host [M, d]) to the device,
  * runs the layer, copies the result into out (host [M, d], out_dtype) and synchronises the
- * stream before returning.  Pinned host memory makes the copies asynchronous to
- * other streams but is not required. */
+ * before returning.  With pinned (page-locked) buffers the copies and kernels are
+ * captured once per (M, k, B, buffer pair) into a CUDA graph on an internal stream
+ * and replayed with one launch; work already queued on `stream` is waited for
+ * first.  Pageable buffers take a plain copy-launch-copy path on `stream`. */
 int moespec_verify_layer_host(moespec_layer_t *layer, const void *hidden_host, int M, int k, int B,
                               void *out_host, void *stream);
 

@@ -24,6 +24,14 @@ struct moespec_layer {
   int last_launches;
   bool profiling;
   cudaEvent_t ev[kMaxProfiled + 1];
+  // host-buffer entry point: the copy-in, the kernels and the copy-out as one instantiated graph
+  cudaStream_t own_stream;
+  cudaEvent_t ev_in;
+  cudaGraphExec_t host_exec;
+  int hg_M, hg_k, hg_B;
+  const void *hg_in;
+  void *hg_out;
+  bool graph_usable;
 };
 
 namespace {
@@ -131,6 +139,15 @@ int validate_call(moespec_layer *L, int M, int k, int B) {
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool is_pinned(const void *p) {
+  cudaPointerAttributes at;
+  if (cudaPointerGetAttributes(&at, p) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  return at.type == cudaMemoryTypeHost;
+}
 
 int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream};
@@ -243,6 +260,9 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
     }
   }
   L->profiling = false;
+  L->host_exec = nullptr;
+  L->graph_usable = cudaStreamCreateWithFlags(&L->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; i <= kMaxProfiled; ++i) {
     e = cudaEventCreate(&L->ev[i]);
     if (e != cudaSuccess) {
@@ -284,11 +304,54 @@ int moespec_verify_layer_host(moespec_layer_t *L, const void *hidden_host, int M
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const size_t bytes = (size_t)M * L->desc.d * elt_bytes(L->desc);
-  cudaError_t e = cudaMemcpyAsync(L->ws.hidden_stage, hidden_host, bytes, cudaMemcpyHostToDevice, s);
+  const size_t out_bytes = (size_t)M * L->desc.d * out_elt_bytes(L->desc);
+  cudaError_t e;
+
+  // Fast path: pinned buffers.  The copy-in, the kernels and the copy-out are captured once per
+  // (M, k, B, buffers) into a graph on an internal stream and replayed with a single launch.
+  if (L->graph_usable && !L->profiling && is_pinned(hidden_host) && is_pinned(out_host)) {
+    const bool hit = L->host_exec && L->hg_M == M && L->hg_k == k && L->hg_B == B && L->hg_in == hidden_host &&
+                     L->hg_out == out_host;
+    if (!hit) {
+      if (L->host_exec) {
+        cudaGraphExecDestroy(L->host_exec);
+        L->host_exec = nullptr;
+      }
+      cudaGraph_t graph = nullptr;
+      e = cudaStreamBeginCapture(L->own_stream, cudaStreamCaptureModeThreadLocal);
+      if (e == cudaSuccess) {
+        e = cudaMemcpyAsync(L->ws.hidden_stage, hidden_host, bytes, cudaMemcpyHostToDevice, L->own_stream);
+        if (e == cudaSuccess && run_layer(L, L->ws.hidden_stage, M, k, B, L->ws.out_stage, L->own_stream) != MOESPEC_OK)
+          e = cudaErrorUnknown;
+        if (e == cudaSuccess)
+          e = cudaMemcpyAsync(out_host, L->ws.out_stage, out_bytes, cudaMemcpyDeviceToHost, L->own_stream);
+        cudaError_t e2 = cudaStreamEndCapture(L->own_stream, &graph);
+        if (e == cudaSuccess) e = e2;
+      }
+      if (e == cudaSuccess) e = cudaGraphInstantiate(&L->host_exec, graph, 0);
+      if (graph) cudaGraphDestroy(graph);
+      if (e != cudaSuccess) {          // graphs unavailable here: use the plain path from now on
+        cudaGetLastError();
+        L->host_exec = nullptr;
+        L->graph_usable = false;
+      } else {
+        L->hg_M = M; L->hg_k = k; L->hg_B = B; L->hg_in = hidden_host; L->hg_out = out_host;
+      }
+    }
+    if (L->host_exec) {
+      // work already queued on the caller's stream (e.g. a weight update) is waited for first
+      if ((e = cudaEventRecord(L->ev_in, s)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaStreamWaitEvent(L->own_stream, L->ev_in, 0)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaGraphLaunch(L->host_exec, L->own_stream)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaStreamSynchronize(L->own_stream)) != cudaSuccess) return cuda_fail(e);
+      return MOESPEC_OK;
+    }
+  }
+
+  e = cudaMemcpyAsync(L->ws.hidden_stage, hidden_host, bytes, cudaMemcpyHostToDevice, s);
   if (e != cudaSuccess) return cuda_fail(e);
   rc = run_layer(L, L->ws.hidden_stage, M, k, B, L->ws.out_stage, s);
   if (rc) return rc;
-  const size_t out_bytes = (size_t)M * L->desc.d * out_elt_bytes(L->desc);
   e = cudaMemcpyAsync(out_host, L->ws.out_stage, out_bytes, cudaMemcpyDeviceToHost, s);
   if (e != cudaSuccess) return cuda_fail(e);
   e = cudaStreamSynchronize(s);
@@ -431,6 +494,11 @@ int moespec_destroy(moespec_layer_t *L) {
   {
     DeviceGuard guard(L->desc.device);
     for (int i = 0; i <= kMaxProfiled; ++i) cudaEventDestroy(L->ev[i]);
+    if (L->host_exec) cudaGraphExecDestroy(L->host_exec);
+    if (L->graph_usable) {
+      cudaEventDestroy(L->ev_in);
+      cudaStreamDestroy(L->own_stream);
+    }
     cudaError_t e = cudaFree(L->arena);
     if (e != cudaSuccess) rc = cuda_fail(e);
   }
