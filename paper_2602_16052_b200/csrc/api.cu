@@ -92,7 +92,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.base = base;
   Workspace w{};
   const size_t N = d.n_experts, M = d.max_M, K = d.max_k, eb = elt_bytes(d);
-  const size_t tiles_up = d.f / kTile + 1, tiles_down = d.d / kTile + 1;
+  const size_t tiles_up = d.f / 32 + 1, tiles_down = d.d / 32 + 1;      // smallest slab height is 32 rows
   // every expert can add at most one partial token chunk beyond the full ones
   const size_t max_chunks = (size_t)R_cap / kMaxTokChunk + N;
   c.take(w.logits, M * N);
@@ -150,7 +150,8 @@ bool is_pinned(const void *p) {
 }
 
 int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
-  LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream};
+  LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
+  if (L->use_tc) c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
   int launches = 0;
   cudaError_t e;
   // with profiling on, an event is recorded before the first kernel and after every kernel
@@ -368,7 +369,8 @@ int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, in
   DeviceGuard guard(L->desc.device);
   if (guard.err != cudaSuccess) return cuda_fail(guard.err);
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap,
-              static_cast<cudaStream_t>(stream)};
+              static_cast<cudaStream_t>(stream), 0};
+  if (L->use_tc) c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
   cudaError_t e = launch_route(c, logits);
   if (e != cudaSuccess) return cuda_fail(e);
   L->last_M = M;

@@ -1,10 +1,14 @@
 // Tensor-core expert FFN for bf16: the weight-streaming kernel of the layer.
 //
-// Work unit = one 128-row slab of one kept expert's weight matrix against one
-// chunk (<= 256) of that expert's routed rows.  Weights are the MMA A operand
-// (rows of W on the M axis, so every weight byte is read from HBM exactly once),
+// Work unit = one slab of RU (128, 64 or 32) rows of one kept expert's weight
+// matrix against one chunk (<= 128) of that expert's routed rows.  RU is chosen
+// per call so that there are a few units per SM even when few experts are kept
+// (small budgets, small trees): an SM can only stream ~55-100 GB/s, so HBM is
+// only saturated when every SM has work.  Weights are the MMA A operand (rows of
+// W on the M axis; the MMA is always M = 128 and rows beyond RU are ignored),
 // routed token rows are the B operand (N axis, padded to a multiple of 32),
-// fp32 accumulators live in tensor memory.
+// fp32 accumulators live in tensor memory (two buffers, so the epilogue of one
+// unit overlaps the MMAs of the next).
 //
 //   gate/up unit:  D_g = W1[e, slab, :] X_e^T,  D_u = W3[e, slab, :] X_e^T,
 //                  h_mid[row, slab] = bf16(silu(D_g) * D_u)
@@ -20,10 +24,11 @@
 // down unit waits for is already running or done: there is no circular wait.
 //
 // Six warps per CTA:
-//   warp 0  lane 0: dispenser + TMA producer.  Streams 64-wide K chunks of the
+//   warp 0        : dispenser + TMA producer.  Lane 0 waits and draws units; all
+//                   lanes issue the copies of a stage: 64-wide K chunks of the
 //                   weight slab(s) (3-D tensor map, expert id is the outer
 //                   coordinate: no stacking copy) and of the token rows into a
-//                   ring of stages, 32 KB of weights per stage.
+//                   ring of stages, up to 32 KB of weights per stage.
 //   warp 1  lane 0: issues tcgen05.mma (kind::f16, M=128, N=n_pad, K=16) from the
 //                   stage's swizzled shared memory into TMEM; tcgen05.commit frees
 //                   the stage and finally publishes the accumulator.
@@ -33,6 +38,7 @@
 // MOESPEC_ERR_TIMEOUT in the status word, drains its own copies, frees TMEM and
 // returns.
 #include "internal.h"
+#include <cstdlib>
 
 namespace moespec {
 
@@ -40,8 +46,9 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kChunkK = 64;                      // bf16 elements per 128-byte swizzle row
-constexpr int kABytes = kTile * kChunkK * 2;     // 16 KB: one weight slab chunk
-constexpr int kBOffset = 2 * kABytes;            // token rows start after two weight chunks
+constexpr int kARegion = 32 * 1024;              // weight bytes per stage
+constexpr int kBRegionMax = 16 * 1024;           // token-row bytes per stage: 8 KB when M <= 32, else 16 KB
+constexpr int kMmaTail = 16 * 1024;              // an M=128 MMA reads 16 KB from the start of a (possibly shorter) slab
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kCtrlBytes = 512;                  // barriers, unit queue, TMEM base, abort flag
@@ -56,13 +63,12 @@ struct TcArgs {
   int *unit_counter;    // dispenser
   int *ready;           // per (expert, token chunk): finished gate/up units
   int tiles_up;         // gate/up units per chunk = value of ready[] that releases its down units
-  int k_iters_up;       // ring stages per gate/up unit: d / 64 (one K chunk of gate and of up per stage)
-  int k_iters_down;     // ring stages per down unit: f / 128 (two K chunks) or f / 64 (one)
-  int down_double;      // 1: a down stage carries two K chunks
-  int b1_off;           // offset of the second token slab inside a stage
+  int ru;               // weight rows per unit: 128, 64 or 32
+  int kchunks_up;       // d / 64: K chunks of a gate/up unit
+  int kchunks_down;     // f / 64: K chunks of a down unit
   int n_stages;
-  int stage_bytes;
-  int acc_bufs;         // 1 or 2 accumulator buffers of 256 TMEM columns
+  int b_region;         // token-row bytes per stage
+  int stage_bytes;      // kARegion + b_region
   __nv_bfloat16 *h_mid; // [R, f]
   float *y;             // [R, d]
   int f, d;
@@ -172,6 +178,19 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
 
 }  // namespace
 
+// K chunks carried by one ring stage of a unit: as many as fit the 32 KB weight region (gate and up
+// slabs in a gate/up unit) and the 16 KB token region (n_pad rows per chunk), a power of two that
+// divides the unit's chunk count.  Producer, MMA issuer and epilogue all derive it from the unit.
+__device__ __forceinline__ int chunks_per_stage(const TcArgs &a, int phase, int n_pad) {
+  const int cap_a = kARegion / ((phase == 0 ? 2 : 1) * a.ru * 128);
+  const int cap_b = a.b_region / (n_pad * 128);
+  const int cap = cap_a < cap_b ? cap_a : cap_b;
+  const int kch = phase == 0 ? a.kchunks_up : a.kchunks_down;
+  int p = 1;
+  while (p * 2 <= cap && kch % (p * 2) == 0) p *= 2;
+  return p;
+}
+
 __device__ __forceinline__ int ld_acquire(const int *p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -180,13 +199,13 @@ __device__ __forceinline__ int ld_acquire(const int *p) {
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMaps maps, TcArgs a) {
+__global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMapsCall maps, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // stages first (1024-byte aligned for the 128-byte swizzle), control block after
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t *smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t ctrl = smem_base + (uint32_t)a.n_stages * (uint32_t)a.stage_bytes;
-  uint8_t *ctrl_gen = smem_gen + (size_t)a.n_stages * a.stage_bytes;
+  const uint32_t ctrl = smem_base + (uint32_t)a.n_stages * (uint32_t)a.stage_bytes + kMmaTail;
+  uint8_t *ctrl_gen = smem_gen + (size_t)a.n_stages * a.stage_bytes + kMmaTail;
   const uint32_t bar_full = ctrl;                       // [kMaxStages]
   const uint32_t bar_empty = ctrl + 8 * kMaxStages;     // [kMaxStages]
   const uint32_t bar_acc_full = ctrl + 16 * kMaxStages; // [2]
@@ -232,71 +251,92 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   // everything above overlaps the tail of the previous kernel; its results are read from here on
   pdl_wait();
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0) {
     // ===================================================== dispenser + TMA producer
+    // Lane 0 owns every wait and the queue; the copies of a stage are issued by all lanes (one box
+    // each), because a single thread issuing 8-16 copies per stage would cap the SM's streaming rate.
+    // CTA b starts with unit b; later units come from the dispenser.  The next unit is drawn a few
+    // stages before the current one ends: early enough that the atomic and the descriptor load are
+    // hidden behind the stages still in flight, late enough that no CTA sits on units others could run.
     const int n_up = a.n_units[0], n_total = n_up + a.n_units[1];
     uint32_t it = 0, qi = 0;
-    bool ok = true;
+    int ok = 1;
     const uint64_t wpol = l2_evict_first_policy();
-    int u = atomicAdd(a.unit_counter, 1);
-    while (ok) {
-      const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
-      if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag)) { ok = false; break; }
-      Unit un;
-      if (u < n_total) {
-        un = a.units[u];
-      } else {
-        un.expert = -1; un.tile = 0; un.row0 = 0; un.n_rows = 0; un.chunk = 0; un.phase = 0; un.pad0 = 0; un.pad1 = 0;
-      }
-      q_unit[q] = un;
-      mbar_arrive(bar_q_full + 8 * q);          // release: the queue slot is visible to the consumers
-      ++qi;
-      if (un.expert < 0) break;
-      const int u_next = atomicAdd(a.unit_counter, 1);   // in flight while this unit streams
-      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
-      if (un.phase == 1) {
-        // the rows of h_mid this unit reads are complete once every gate/up slab of the chunk is done
-        const long long t0 = clock64();
-        while (ld_acquire(a.ready + un.chunk) < a.tiles_up) {
-          if (*abort_flag || clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; ok = false; break; }
-          __nanosleep(64);
+    Unit sentinel;
+    sentinel.expert = -1; sentinel.tile = 0; sentinel.row0 = 0; sentinel.n_rows = 0; sentinel.chunk = 0;
+    sentinel.phase = 0; sentinel.pad0 = 0; sentinel.pad1 = 0;
+    Unit un = sentinel;
+    if (lane == 0 && (int)blockIdx.x < n_total) un = a.units[blockIdx.x];
+    while (true) {
+      Unit un_next = sentinel;
+      int u_next = n_total;
+      if (lane == 0) {
+        const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
+        if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag)) ok = 0;
+        if (ok) {
+          q_unit[q] = un;
+          mbar_arrive(bar_q_full + 8 * q);          // release: the queue slot is visible to the consumers
+          if (un.expert >= 0 && un.phase == 1) {
+            // the rows of h_mid this unit reads are complete once every gate/up slab of the chunk is done
+            const long long t0 = clock64();
+            while (ld_acquire(a.ready + un.chunk) < a.tiles_up) {
+              if (*abort_flag || clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; ok = 0; break; }
+              __nanosleep(64);
+            }
+            fence_proxy_async();                    // order the acquire before the TMA reads of h_mid
+          }
         }
-        if (!ok) break;
-        fence_proxy_async();                    // order the acquire before the TMA reads of h_mid
       }
-      const int k_iters = un.phase == 0 ? a.k_iters_up : a.k_iters_down;
-      const CUtensorMap *map_b = un.phase == 0 ? &maps.x_perm : &maps.h_mid;
+      ++qi;
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      const int expert = __shfl_sync(0xffffffffu, un.expert, 0);
+      if (!ok || expert < 0) break;
+      const int tile = __shfl_sync(0xffffffffu, un.tile, 0);
+      const int row0 = __shfl_sync(0xffffffffu, un.row0, 0);
+      const int n_rows = __shfl_sync(0xffffffffu, un.n_rows, 0);
+      const int phase = __shfl_sync(0xffffffffu, un.phase, 0);
+      const int n_pad = (n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const int cps = chunks_per_stage(a, phase, n_pad);
+      const int k_iters = (phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
+      const uint32_t slab_bytes = (uint32_t)n_pad * 128u;           // one K chunk of the unit's token rows
+      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm : &maps.h_mid;
+      const uint32_t sub_bytes = (uint32_t)a.ru * 128u;            // one K chunk of one weight slab
+      const int w_boxes = (phase == 0 ? 2 : 1) * cps;              // weight copies per stage
+      const int t_per = n_pad / kTokBox;                           // token copies per K chunk
+      const int n_boxes = w_boxes + cps * t_per;
+      const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_pad * 128u;
+      const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
-        if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t full = bar_full + 8 * s;
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
-        if (un.phase == 0) {
-          mbar_expect_tx(full, 2u * kABytes + (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_gate, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
-          tma_load_3d(stage + kABytes, &maps.w_up, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
-          for (int b = 0; b < n_pad / kTokBox; ++b)
-            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
-        } else if (a.down_double) {
-          mbar_expect_tx(full, 2u * kABytes + 2u * (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_down, full, (2 * kc) * kChunkK, un.tile * kTile, un.expert, wpol);
-          tma_load_3d(stage + kABytes, &maps.w_down, full, (2 * kc + 1) * kChunkK, un.tile * kTile, un.expert, wpol);
-          for (int b = 0; b < n_pad / kTokBox; ++b) {
-            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, (2 * kc) * kChunkK, un.row0 + b * kTokBox);
-            tma_load_2d(stage + a.b1_off + b * (kTokBox * 128), map_b, full, (2 * kc + 1) * kChunkK,
-                        un.row0 + b * kTokBox);
+        if (lane == 0) {
+          if (kc == draw_at) u_next = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
+          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) ok = 0;
+          else mbar_expect_tx(full, tx);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        for (int b = lane; b < n_boxes; b += 32) {
+          if (b < w_boxes) {
+            const int j = phase == 0 ? (b >> 1) : b;
+            const int col = (kc * cps + j) * kChunkK;
+            const CUtensorMap *mw = phase == 0 ? ((b & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
+            tma_load_3d(stage + b * sub_bytes, mw, full, col, tile * a.ru, expert, wpol);
+          } else {
+            const int tb = b - w_boxes;
+            const int j = tb / t_per, r = tb - j * t_per;
+            const int col = (kc * cps + j) * kChunkK;
+            tma_load_2d(stage + kARegion + j * slab_bytes + r * (kTokBox * 128), map_b, full, col, row0 + r * kTokBox);
           }
-        } else {
-          mbar_expect_tx(full, (uint32_t)kABytes + (uint32_t)n_pad * 128u);
-          tma_load_3d(stage, &maps.w_down, full, kc * kChunkK, un.tile * kTile, un.expert, wpol);
-          for (int b = 0; b < n_pad / kTokBox; ++b)
-            tma_load_2d(stage + kBOffset + b * (kTokBox * 128), map_b, full, kc * kChunkK, un.row0 + b * kTokBox);
         }
       }
-      u = u_next;
+      if (!ok) break;
+      if (lane == 0 && u_next < n_total) un_next = a.units[u_next];
+      un = un_next;
     }
-    if (!ok) {
-      // drain: wait (bounded) until every copy this thread issued has landed
+    if (!ok && lane == 0) {
+      // drain: wait (bounded) until every copy this warp issued has landed
       const uint32_t lo = it > (uint32_t)n_stages ? it - n_stages : 0u;
       for (uint32_t j = lo; j < it; ++j) {
         const long long t0 = clock64();
@@ -316,33 +356,45 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t idesc = instr_desc_bf16(n_pad);
-      const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
+      const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
       if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) break;
       tc_fence_after();
       const uint32_t tmem_d = tmem_base + ab * 256u;
-      const int k_iters = un.phase == 0 ? a.k_iters_up : a.k_iters_down;
+      const int cps = chunks_per_stage(a, un.phase, n_pad);
+      const int k_iters = (un.phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
+      // This one thread issues every MMA of the CTA, so its instruction count per MMA bounds the rate at
+      // which stages are released.  Descriptors are therefore advanced by adding to the 16-byte-granular
+      // address field instead of being rebuilt: +2 per K step of 16 elements, +sub16 per weight slab,
+      // +slab16 per token slab.
+      const uint64_t sub16 = (uint64_t)(a.ru * 128 >> 4), slab16 = (uint64_t)(n_pad * 128 >> 4);
+      const uint32_t tmem_u = tmem_d + (uint32_t)n_pad;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
+        uint64_t ad = smem_desc_sw128(smem_base + s * (uint32_t)a.stage_bytes);
+        uint64_t bd = ad + (uint64_t)(kARegion >> 4);
+        uint32_t acc = kc > 0 ? 1u : 0u;
         if (un.phase == 0) {
+          for (int j = 0; j < cps; ++j) {
 #pragma unroll
-          for (int kk = 0; kk < kChunkK / 16; ++kk) {
-            const uint32_t acc = (kc > 0 || kk > 0) ? 1u : 0u;
-            const uint64_t bdesc = smem_desc_sw128(stage + kBOffset + kk * 32);
-            tc_mma_bf16(tmem_d, smem_desc_sw128(stage + kk * 32), bdesc, idesc, acc);
-            tc_mma_bf16(tmem_d + (uint32_t)n_pad, smem_desc_sw128(stage + kABytes + kk * 32), bdesc, idesc, acc);
+            for (int kk = 0; kk < kChunkK / 16; ++kk) {
+              tc_mma_bf16(tmem_d, ad + 2 * kk, bd + 2 * kk, idesc, acc);
+              tc_mma_bf16(tmem_u, ad + sub16 + 2 * kk, bd + 2 * kk, idesc, acc);
+              acc = 1u;
+            }
+            ad += 2 * sub16;
+            bd += slab16;
           }
         } else {
-          const int halves = a.down_double ? 2 : 1;
-          for (int half = 0; half < halves; ++half) {
-            const uint32_t a_off = stage + half * kABytes;
-            const uint32_t b_off = stage + (half ? (uint32_t)a.b1_off : (uint32_t)kBOffset);
+          for (int j = 0; j < cps; ++j) {
 #pragma unroll
-            for (int kk = 0; kk < kChunkK / 16; ++kk)
-              tc_mma_bf16(tmem_d, smem_desc_sw128(a_off + kk * 32), smem_desc_sw128(b_off + kk * 32), idesc,
-                          (kc > 0 || half > 0 || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < kChunkK / 16; ++kk) {
+              tc_mma_bf16(tmem_d, ad + 2 * kk, bd + 2 * kk, idesc, acc);
+              acc = 1u;
+            }
+            ad += sub16;
+            bd += slab16;
           }
         }
         tc_commit(bar_empty + 8 * s);      // stage reusable once these MMAs have read it
@@ -363,13 +415,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const Unit un = q_unit[q];
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
-      const uint32_t ab = acc_it % a.acc_bufs, aph = (acc_it / a.acc_bufs) & 1u;
+      const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
       if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag)) break;
       tc_fence_after();
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
-      const int col_out = un.tile * kTile + row_in_tile;    // index along f (gate/up) or d (down)
-      for (int c0 = 0; c0 < un.n_rows; c0 += 16) {
+      const int col_out = un.tile * a.ru + row_in_tile;     // index along f (gate/up) or d (down)
+      const int n_live = quarter * 32 < a.ru ? un.n_rows : 0;   // accumulator lanes beyond RU hold nothing
+      for (int c0 = 0; c0 < n_live; c0 += 16) {
         uint32_t g[16];
         tc_ld16(taddr + c0, g);
         if (un.phase == 0) {
@@ -434,10 +487,10 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
   cudaError_t e = get_encode_fn(&enc);
   if (e != cudaSuccess) return e;
   const cuuint32_t ones[3] = {1, 1, 1};
-  auto weights = [&](CUtensorMap *m, const void *base, int rows, int K) -> CUresult {
+  auto weights = [&](CUtensorMap *m, const void *base, int rows, int K, int box_rows) -> CUresult {
     cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)d.n_experts};
     cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)rows * K * 2};
-    cuuint32_t box[3] = {kChunkK, kTile, 1};
+    cuuint32_t box[3] = {kChunkK, (cuuint32_t)box_rows, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, ones,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -449,12 +502,16 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   };
-  CUresult r;
-  if ((r = weights(&maps->w_gate, d.w_gate, d.f, d.d)) != CUDA_SUCCESS ||
-      (r = weights(&maps->w_up, d.w_up, d.f, d.d)) != CUDA_SUCCESS ||
-      (r = weights(&maps->w_down, d.w_down, d.d, d.f)) != CUDA_SUCCESS ||
-      (r = rows2d(&maps->x_perm, ws.x_perm, d.d)) != CUDA_SUCCESS ||
-      (r = rows2d(&maps->h_mid, ws.h_mid, d.f)) != CUDA_SUCCESS) {
+  CUresult r = CUDA_SUCCESS;
+  for (int i = 0; i < 3 && r == CUDA_SUCCESS; ++i) {
+    const int box_rows = kTile >> i;      // 128, 64, 32
+    if ((r = weights(&maps->w_gate[i], d.w_gate, d.f, d.d, box_rows)) != CUDA_SUCCESS) break;
+    if ((r = weights(&maps->w_up[i], d.w_up, d.f, d.d, box_rows)) != CUDA_SUCCESS) break;
+    r = weights(&maps->w_down[i], d.w_down, d.d, d.f, box_rows);
+  }
+  if (r == CUDA_SUCCESS) r = rows2d(&maps->x_perm, ws.x_perm, d.d);
+  if (r == CUDA_SUCCESS) r = rows2d(&maps->h_mid, ws.h_mid, d.f);
+  if (r != CUDA_SUCCESS) {
     *cu_result = (int)r;
     return cudaErrorInvalidValue;
   }
@@ -474,31 +531,49 @@ static int sm_count_cached(int device) {
   return n;
 }
 
+int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
+  // Measured on B200: 128-row slabs stream fastest (each unit re-reads its expert's token rows, so
+  // shorter slabs double the L2->SM traffic per weight byte); 64-row slabs only pay off when there would
+  // otherwise be fewer gate/up units than half the SMs (a handful of kept experts, e.g. M = 1).
+  int active = B < D.n_experts ? B : D.n_experts;          // upper bound of kept experts that get rows
+  if ((long long)M * k < active) active = M * k;
+  static const int forced = [] { const char *v = getenv("MOESPEC_FORCE_RU"); return v ? atoi(v) : 0; }();
+  if (forced == 128 || forced == 64 || forced == 32) return forced;     // experiments only
+  return (long long)active * (D.f / kTile) * 2 < sm_count_cached(D.device) ? 64 : kTile;
+}
+
 cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps) {
   const moespec_layer_desc &D = *c.desc;
-  const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
+  const int ru = c.ru;
+  const int ri = ru == 128 ? 0 : ru == 64 ? 1 : 2;
   TcArgs a;
-  a.down_double = n_pad_max <= 128 ? 1 : 0;      // two K chunks per down stage while both token slabs fit
-  a.b1_off = kBOffset + n_pad_max * 128;
-  a.stage_bytes = kBOffset + (a.down_double ? 2 : 1) * n_pad_max * 128;
-  int stages = (kSmemBudget - 1024 - kCtrlBytes) / a.stage_bytes;
+  a.ru = ru;
+  a.kchunks_up = D.d / kChunkK;
+  a.kchunks_down = D.f / kChunkK;
+  const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
+  a.b_region = n_pad_max * 128 * 2 < kBRegionMax ? n_pad_max * 128 * 2 : kBRegionMax;
+  a.stage_bytes = kARegion + a.b_region;
+  int stages = (kSmemBudget - 1024 - kCtrlBytes - kMmaTail) / a.stage_bytes;
   a.n_stages = stages > kMaxStages ? kMaxStages : stages;
-  a.acc_bufs = 2 * n_pad_max <= 256 ? 2 : 1;
   a.status = c.ws->status;
   a.units = c.ws->units;
   a.n_units = c.ws->counters + 3;
   a.unit_counter = c.ws->unit_counter;
   a.ready = c.ws->ready;
-  a.tiles_up = D.f / kTile;
-  a.k_iters_up = D.d / kChunkK;
-  a.k_iters_down = a.down_double ? D.f / (2 * kChunkK) : D.f / kChunkK;
+  a.tiles_up = D.f / ru;
   a.h_mid = reinterpret_cast<__nv_bfloat16 *>(c.ws->h_mid);
   a.y = c.ws->y;
   a.f = D.f;
   a.d = D.d;
+  TcMapsCall m;
+  m.w_gate = maps->w_gate[ri];
+  m.w_up = maps->w_up[ri];
+  m.w_down = maps->w_down[ri];
+  m.x_perm = maps->x_perm;
+  m.h_mid = maps->h_mid;
   const int grid = sm_count_cached(D.device);
-  const size_t smem = (size_t)a.n_stages * a.stage_bytes + 1024 + kCtrlBytes;
-  return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, *maps, a);
+  const size_t smem = (size_t)a.n_stages * a.stage_bytes + kMmaTail + 1024 + kCtrlBytes;
+  return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, m, a);
 }
 
 }  // namespace moespec

@@ -13,10 +13,10 @@ constexpr int kMaskWords = kMaxExperts / 32;
 constexpr int kMaxK = 32;
 constexpr int kTile = 128;                 // weight rows per tensor-core work unit (MMA M)
 constexpr int kTokBox = 32;                // token rows per TMA box of the B operand
-constexpr int kMaxTokChunk = 256;          // tokens per work unit (MMA N limit)
+constexpr int kMaxTokChunk = 128;          // tokens per work unit: gate and up accumulators of two units fit TMEM
 
-// One tensor-core work unit: a 128-row slab of one expert's weight matrix
-// against one chunk (<= 256) of that expert's routed rows.
+// One tensor-core work unit: a slab of RU (128, 64 or 32) rows of one expert's weight
+// matrix against one chunk (<= 128) of that expert's routed rows.
 struct __align__(16) Unit {
   int expert;
   int tile;       // slab index along f (gate/up phase) or d (down phase)
@@ -70,6 +70,7 @@ struct LaunchCtx {
   int M, k, B;
   int R_cap;            // max_M * max_k
   cudaStream_t stream;
+  int ru;               // weight rows per tensor-core work unit for this call (0: CUDA-core path)
 };
 
 // Programmatic dependent launch.  Every kernel of the layer is launched with
@@ -109,9 +110,13 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
 // ffn_simple.cu
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down
 // ffn_tc.cu
-struct TcMaps {
+struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 32
+  CUtensorMap w_gate[3], w_up[3], w_down[3], x_perm, h_mid;
+};
+struct TcMapsCall {        // per launch: the maps of the chosen slab height
   CUtensorMap w_gate, w_up, w_down, x_perm, h_mid;
 };
+int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // slab height for a call
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes

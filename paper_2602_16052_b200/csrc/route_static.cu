@@ -123,6 +123,6 @@ extern "C" int moespec_route_static(const float *logits, int M, int N, int k, in
   desc.policy = policy;
   desc.shortlist = shortlist;
   desc.renormalize = renormalize;
-  LaunchCtx c{&desc, &ws, M, k, B > N ? N : B, M * k, static_cast<cudaStream_t>(stream)};
+  LaunchCtx c{&desc, &ws, M, k, B > N ? N : B, M * k, static_cast<cudaStream_t>(stream), 0};
   return launch_route(c, logits) == cudaSuccess ? MOESPEC_OK : MOESPEC_ERR_CUDA;
 }

@@ -291,7 +291,7 @@ struct RouteArgs {
   Workspace ws;
   int M, N, k, B;
   int policy, shortlist, renormalize;
-  int tiles_up, tiles_down;     // f/128, d/128 (0 when the tensor-core path is not used)
+  int tiles_up, tiles_down;     // f/RU, d/RU slabs per expert (0 when the tensor-core path is not used)
   long long expert_bytes;       // 3*d*f*sizeof(dtype)
 };
 
@@ -579,18 +579,22 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         const int phase = u >= n_up;
         const int tiles = phase ? a.tiles_down : a.tiles_up;
         const int v = phase ? u - n_up : u;
-        const int ci = v / tiles, tl = v - ci * tiles;
+        const int cpos = v / tiles;           // position in chunk-prefix space: identifies the expert
         int e;
-        if (ci < 2 * kMaxExperts) {
-          e = s_chunk_expert[ci];
-        } else {          // more than 2N token chunks (M far beyond 256): search the chunk bases
+        if (cpos < 2 * kMaxExperts) {
+          e = s_chunk_expert[cpos];
+        } else {          // more than 2N token chunks (M far beyond 128): search the chunk bases
           e = 0;
-          while (s_unit_base[e + 1] <= ci) ++e;
+          while (s_unit_base[e + 1] <= cpos) ++e;
         }
-        const int c = ci - s_unit_base[e];
+        // inside an expert: slab-major, token chunk innermost, so the chunks that re-read a slab are
+        // handed out back to back and the second read hits L2
+        const int chunks_e = s_unit_base[e + 1] - s_unit_base[e];
+        const int local = v - s_unit_base[e] * tiles;
+        const int tl = local / chunks_e, c = local - tl * chunks_e;
         const int row0 = s_offset[e] + c * kMaxTokChunk;
         const int rows = min(kMaxTokChunk, s_count[e] - c * kMaxTokChunk);
-        ws.units[u] = Unit{e, tl, row0, rows, ci, phase, 0, 0};
+        ws.units[u] = Unit{e, tl, row0, rows, s_unit_base[e] + c, phase, 0, 0};
       }
     }
   } else {
@@ -646,9 +650,8 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.ws = *c.ws;
   a.M = c.M; a.N = D.n_experts; a.k = c.k; a.B = c.B;
   a.policy = D.policy; a.shortlist = D.shortlist; a.renormalize = D.renormalize;
-  const bool tc = (D.f % kTile == 0) && (D.d % kTile == 0);
-  a.tiles_up = tc ? D.f / kTile : 0;
-  a.tiles_down = tc ? D.d / kTile : 0;
+  a.tiles_up = c.ru > 0 ? D.f / c.ru : 0;
+  a.tiles_down = c.ru > 0 ? D.d / c.ru : 0;
   a.expert_bytes = 3LL * D.d * D.f * (D.dtype == MOESPEC_BF16 ? 2 : 4);
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
