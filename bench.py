@@ -244,6 +244,20 @@ def run_tables(args, device):
         torch.cuda.empty_cache()
 
 
+def job_time_ms(local_ms: float, dist=None, device=None) -> float:
+    """Job time of a replicated run: the slowest rank's device time (max over ranks)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return local_ms
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_us_per_layer(job_ms: float, steps: int, world: int) -> float:
+    """Whole-job metric of N independent replicas: every rank ran `steps` layers in `job_ms`."""
+    return job_ms * 1e3 / (steps * world)
+
+
 def oracle_case(cfg, M, seed):
     L = synth.gen_layer(cfg, seed=seed, layer=0, device="cpu")
     h = synth.gen_hidden(cfg, M, seed=seed, layer=0, device="cpu")
@@ -331,11 +345,7 @@ def main():
             dist.barrier()
 
     def max_over_ranks(x: float) -> float:
-        if dist is None:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return job_time_ms(x, dist, device)
 
     if args.tables:
         return run_tables(args, device)
@@ -369,8 +379,8 @@ def main():
     e2e_ms = max_over_ranks(e2e_ms)
 
     # value: job-wide microseconds per verify layer (all ranks' layers / max time over ranks)
-    us_per_layer = ms_total * 1e3 / (args.steps * world)
-    e2e_us = e2e_ms * 1e3 / (args.steps * world)
+    us_per_layer = job_us_per_layer(ms_total, args.steps, world)
+    e2e_us = job_us_per_layer(e2e_ms, args.steps, world)
 
     # roofline of the dominant kernel: the expert-FFN weight stream (two launches of ffn_tc_kernel per layer)
     peak, peak_kind = measured_peaks()

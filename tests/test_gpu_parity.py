@@ -25,6 +25,8 @@ def ms():
 
 
 def make_layer(case, max_M, max_k, **kw):
+    kw.setdefault("policy", ms().SUBSTITUTION)
+    kw.setdefault("shortlist", ms().FROM_ALL)
     return ms().Layer(case["router_w"], case["router_bias"], case["w_gate"], case["w_up"], case["w_down"],
                       max_M=max_M, max_k=max_k, **kw)
 
@@ -40,8 +42,8 @@ def check_out(out, ref, dtype):
         err = float(np.max(np.abs(o - ref)))
         assert err <= BF16_TOL * rms, f"max err {err:.3e} > {BF16_TOL} * rms {rms:.3e}"
     elif dtype == "bf16":
-        # out stored as bf16: the stated bar plus the final rounding of the result itself (half an ulp <= 2^-9 |ref|)
-        bound = BF16_TOL * rms + 2.0 ** -9 * np.abs(ref)
+        # out stored as bf16: the stated bar plus the final rounding of the result itself (half an ulp <= 2^-8 |ref|)
+        bound = BF16_TOL * rms + 2.0 ** -8 * np.abs(ref)
         assert np.all(np.abs(o - ref) <= bound), f"worst {np.max(np.abs(o - ref) / np.maximum(bound, 1e-300)):.2f}x of bound"
     else:
         bound = FP32_TOL * np.maximum(np.abs(ref), rms)
@@ -289,3 +291,31 @@ def test_argument_errors_return_codes():
     with pytest.raises(m.MoeSpecError):
         make_layer(case, max_M=15, max_k=4, ffn_kernel=m.FFN_TENSOR_CORE)    # fp32 has no tensor-core kernel
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ stack of layers (residual, bf16 stream)
+def test_stack_teacher_forced_parity_and_drift():
+    """x <- bf16(x + MoE_l(x)) over independent seeded layers.  Every GPU layer is fed the oracle's
+    input for that layer (pass/fail); the free-running GPU stack's drift is only bounded loosely."""
+    m = ms()
+    cfg = synth.CONFIGS["olmoe"].with_(f=256, n_experts=32, n_layers=4)
+    M, B = 31, 12
+    x_ref = H.f64(synth.gen_hidden(cfg, M, seed=9))
+    x_gpu = synth.gen_hidden(cfg, M, seed=9, device="cuda")
+    for l in range(cfg.n_layers):
+        case = synth.gen_layer(cfg, 9, l, "cuda")
+        layer = make_layer(case, M, cfg.k, residual=True, out_dtype=torch.bfloat16)
+        case["hidden"] = torch.from_numpy(x_ref).to("cuda", torch.bfloat16)       # teacher forcing
+        out = layer.verify_layer(case["hidden"], cfg.k, B)
+        torch.cuda.synchronize()
+        r = H.oracle_run(case, cfg.k, B, orc.SUBSTITUTION, orc.FROM_ALL, True, logits=layer.get_logits())
+        H.compare_routing(layer.get_routing(), r, orc.SUBSTITUTION, cfg.k)
+        nxt = x_ref + r["out"]
+        rms = float(np.sqrt(np.mean(r["out"] ** 2)))
+        bound = BF16_TOL * rms + 2.0 ** -8 * np.abs(nxt)                          # + rounding of the bf16 stream
+        assert np.all(np.abs(H.f64(out) - nxt) <= bound)
+        x_gpu = layer.verify_layer(x_gpu, cfg.k, B).clone()                       # free-running stack
+        x_ref = orc.round_bf16(nxt)                                               # the oracle's stream is bf16 too
+        layer.destroy()
+    drift = np.abs(H.f64(x_gpu) - x_ref).max() / np.sqrt(np.mean(x_ref ** 2))
+    assert drift < 0.25, f"free-running drift {drift:.3f}"
