@@ -206,9 +206,10 @@ int moespec_get_stats(moespec_layer_t *layer, moespec_stats *stats);
  * stream before the first kernel and after every kernel (do not enable it while
  * the stream is being captured into a graph).  get_kernel_times waits for the
  * last verify call and writes the duration in milliseconds of each of its
- * kernels, in launch order (router + softmax + top-k, routing, gather, expert FFN
- * [one launch for bf16 tensor cores; gate/up and down launches for the CUDA-core
- * kernel], combine), into ms[0 .. min(capacity, *n_kernels)). */
+ * kernels, in launch order, into ms[0 .. min(capacity, *n_kernels)).  bf16 tensor-core
+ * layers launch four kernels (router + softmax + top-k; routing; gather; expert FFN +
+ * combine); CUDA-core layers launch six (router, routing, gather, FFN gate/up, FFN
+ * down, combine). */
 int moespec_set_profiling(moespec_layer_t *layer, int on);
 int moespec_get_kernel_times(moespec_layer_t *layer, float *ms, int capacity, int *n_kernels);
 

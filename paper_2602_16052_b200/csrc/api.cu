@@ -166,16 +166,17 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   if (L->use_tc) {
-    if ((e = launch_ffn_tensor_core(c, &L->maps)) != cudaSuccess) return cuda_fail(e);
+    // both FFN phases and the combine are one persistent kernel
+    if ((e = launch_ffn_tensor_core(c, &L->maps, hidden, out)) != cudaSuccess) return cuda_fail(e);
     if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   } else {
     for (int phase = 0; phase < 2; ++phase) {
       if ((e = launch_ffn_cuda_core(c, phase)) != cudaSuccess) return cuda_fail(e);
       if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
     }
+    if ((e = launch_combine(c, hidden, out)) != cudaSuccess) return cuda_fail(e);
+    if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   }
-  if ((e = launch_combine(c, hidden, out)) != cudaSuccess) return cuda_fail(e);
-  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   L->last_M = M;
   L->last_k = k;
   L->last_launches = launches;

@@ -34,6 +34,12 @@
 //                   the stage and finally publishes the accumulator.
 //   warps 2-5     : epilogue.  tcgen05.ld the accumulator (one TMEM lane quarter
 //                   per warp), apply SwiGLU, store to global.
+// The combine of the layer lives in this kernel too: after its last unit every
+// CTA waits (bounded) until all down units are stored and then produces its share
+// of `out` from y, the mixing weights and tokslot2row, adding slots in a fixed
+// order.  (Fetching routed rows straight from `hidden` with one-row TMA boxes was
+// measured 40 % slower than reading a gathered copy with 32-row boxes: the copy
+// engine's rate for 128-byte boxes is the limit.)
 // Every wait is bounded: on expiry the CTA raises an abort flag, records
 // MOESPEC_ERR_TIMEOUT in the status word, drains its own copies, frees TMEM and
 // returns.
@@ -73,6 +79,13 @@ struct TcArgs {
   float *y;             // [R, d]
   int f, d;
   int *status;
+  // combine (outer sums of Eq. 2 / 7 / 8), run by every CTA once all down units are stored
+  int *down_done;       // down units whose y slab is stored; zeroed by the route kernel
+  const float *gate_w;  // [M, k]
+  const int *tokslot2row;
+  const void *hidden;   // [M, d] bf16 (residual input)
+  void *out;            // [M, d] bf16 or fp32
+  int M, k, residual, out_is_fp32;
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -299,12 +312,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int cps = chunks_per_stage(a, phase, n_pad);
       const int k_iters = (phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
       const uint32_t slab_bytes = (uint32_t)n_pad * 128u;           // one K chunk of the unit's token rows
-      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm : &maps.h_mid;
       const uint32_t sub_bytes = (uint32_t)a.ru * 128u;            // one K chunk of one weight slab
       const int w_boxes = (phase == 0 ? 2 : 1) * cps;              // weight copies per stage
-      const int t_per = n_pad / kTokBox;                           // token copies per K chunk
-      const int n_boxes = w_boxes + cps * t_per;
-      const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_pad * 128u;
+      const int t_per = n_pad / kTokBox;                           // 32-row token copies per K chunk
+      const int n_tok_rows = n_pad;                                // rows that arrive per K chunk
+      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm : &maps.h_mid;
+      const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_tok_rows * 128u;
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
@@ -317,18 +330,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        for (int b = lane; b < n_boxes; b += 32) {
-          if (b < w_boxes) {
-            const int j = phase == 0 ? (b >> 1) : b;
-            const int col = (kc * cps + j) * kChunkK;
-            const CUtensorMap *mw = phase == 0 ? ((b & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
-            tma_load_3d(stage + b * sub_bytes, mw, full, col, tile * a.ru, expert, wpol);
-          } else {
-            const int tb = b - w_boxes;
-            const int j = tb / t_per, r = tb - j * t_per;
-            const int col = (kc * cps + j) * kChunkK;
-            tma_load_2d(stage + kARegion + j * slab_bytes + r * (kTokBox * 128), map_b, full, col, row0 + r * kTokBox);
-          }
+        if (lane < w_boxes) {                       // at most 8 weight copies per stage
+          const int j = phase == 0 ? (lane >> 1) : lane;
+          const int col = (kc * cps + j) * kChunkK;
+          const CUtensorMap *mw = phase == 0 ? ((lane & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
+          tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * a.ru, expert, wpol);
+        }
+        for (int tb = lane; tb < cps * t_per; tb += 32) {
+          const int j = tb / t_per, r = tb - j * t_per;
+          const int col = (kc * cps + j) * kChunkK;
+          tma_load_2d(stage + kARegion + j * slab_bytes + r * (kTokBox * 128), map_b, full, col, row0 + r * kTokBox);
         }
       }
       if (!ok) break;
@@ -446,13 +457,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       }
       tc_fence_before();
       mbar_arrive(bar_acc_empty + 8 * ab);
-      if (un.phase == 0) {
-        // publish this slab of h_mid: every thread's stores are fenced, then one thread bumps the counter
-        __threadfence();
-        fence_proxy_async();
-        epilogue_bar();
-        if (threadIdx.x == 64) atomicAdd(a.ready + un.chunk, 1);
-      }
+      // publish the slab (h_mid for a gate/up unit, y for a down unit): every thread's stores are
+      // fenced, then one thread bumps the counter the consumers of the slab watch
+      __threadfence();
+      if (un.phase == 0) fence_proxy_async();
+      epilogue_bar();
+      if (threadIdx.x == 64) atomicAdd(un.phase == 0 ? a.ready + un.chunk : a.down_done, 1);
       mbar_arrive(bar_q_empty + 8 * q);
       ++acc_it;
     }
@@ -460,10 +470,71 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, (int)MOESPEC_ERR_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+
+  // ===================================================== combine
+  // out_t = sum over the kept slots of wgt[t, slot] * y[row(t, slot)], slots in a fixed order; a token
+  // with no kept expert gets exact zeros (Section 3.3).  Needs every down unit of the call.
+  if (threadIdx.x == 0 && !*abort_flag) {
+    const int n_down = a.n_units[1];
+    const long long t0 = clock64();
+    while (ld_acquire(a.down_done) < n_down) {
+      if (clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; break; }
+      __nanosleep(128);
+    }
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    if (threadIdx.x == 0) atomicExch(a.status, (int)MOESPEC_ERR_TIMEOUT);
+    return;
+  }
+  const int k = a.k, d = a.d;
+  // work item = one quarter of one token's columns, so that small trees still spread over the SMs
+  const int qcols = d / 4;
+  for (int item = blockIdx.x; item < a.M * 4; item += gridDim.x) {
+    const int t = item >> 2, c_lo = (item & 3) * qcols;
+    for (int c = c_lo + threadIdx.x * 4; c < c_lo + qcols; c += kThreads * 4) {
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      for (int s0 = 0; s0 < k; s0 += 8) {
+        float4 v[8];
+        float w[8];
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+          const int row = s0 + s < k ? a.tokslot2row[(size_t)t * k + s0 + s] : -1;
+          w[s] = row >= 0 ? a.gate_w[(size_t)t * k + s0 + s] : 0.f;
+          v[s] = row >= 0 ? __ldcg(reinterpret_cast<const float4 *>(a.y + (size_t)row * d + c))
+                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int s = 0; s < 8; ++s) {
+          if (s0 + s < k && w[s] != 0.f) {
+            acc.x = fmaf(w[s], v[s].x, acc.x);
+            acc.y = fmaf(w[s], v[s].y, acc.y);
+            acc.z = fmaf(w[s], v[s].z, acc.z);
+            acc.w = fmaf(w[s], v[s].w, acc.w);
+          }
+        }
+      }
+      if (a.residual) {
+        const uint2 raw = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.hidden) +
+                                                            (size_t)t * d + c);
+        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+        const float2 lo = __bfloat1622float2(h2[0]), hi = __bfloat1622float2(h2[1]);
+        acc.x += lo.x; acc.y += lo.y; acc.z += hi.x; acc.w += hi.y;
+      }
+      if (a.out_is_fp32) {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + (size_t)t * d + c) = acc;
+      } else {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+        uint2 raw;
+        raw.x = *reinterpret_cast<uint32_t *>(&lo);
+        raw.y = *reinterpret_cast<uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + (size_t)t * d + c) = raw;
+      }
+    }
   }
 }
 
@@ -542,7 +613,7 @@ int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
   return (long long)active * (D.f / kTile) * 2 < sm_count_cached(D.device) ? 64 : kTile;
 }
 
-cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps) {
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
   const int ru = c.ru;
   const int ri = ru == 128 ? 0 : ru == 64 ? 1 : 2;
@@ -565,6 +636,15 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps) {
   a.y = c.ws->y;
   a.f = D.f;
   a.d = D.d;
+  a.down_done = c.ws->unit_counter + 1;
+  a.gate_w = c.ws->gate_w;
+  a.tokslot2row = c.ws->tokslot2row;
+  a.hidden = hidden;
+  a.out = out;
+  a.M = c.M;
+  a.k = c.k;
+  a.residual = D.residual;
+  a.out_is_fp32 = (D.out_dtype ? D.out_dtype : D.dtype) == MOESPEC_FP32;
   TcMapsCall m;
   m.w_gate = maps->w_gate[ri];
   m.w_up = maps->w_up[ri];

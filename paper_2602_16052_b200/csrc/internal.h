@@ -53,7 +53,7 @@ struct Workspace {
   int mask_words;       // ceil(max_M / 32)
   Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
   int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
-  int *unit_counter;    // next unit to hand out; zeroed by the route kernel
+  int *unit_counter;    // [0] next unit to hand out, [1] finished down units; zeroed by the route kernel
   int *counters;        // [0]=n_S [1]=n_active [2]=R [3]=n_units_up [4]=n_units_down
   moespec_stats *stats; // device copy
   int *status;          // device status word (0 = ok)
@@ -120,7 +120,8 @@ int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // sla
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes
-cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps);   // both phases, one launch
+// gate/up + down + combine in one launch
+cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const void *hidden, void *out);
 // combine.cu
 cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out);
 

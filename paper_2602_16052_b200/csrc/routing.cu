@@ -574,7 +574,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       const int lt = tid - 128, nthr = 96;
       const int n_up = n_chunks * a.tiles_up, n_down = n_chunks * a.tiles_down;
       for (int i = lt; i < n_chunks; i += nthr) ws.ready[i] = 0;
-      if (lt == 0) *ws.unit_counter = 0;
+      if (lt == 0) {
+        ws.unit_counter[0] = 0;
+        ws.unit_counter[1] = 0;
+      }
       for (int u = lt; u < n_up + n_down; u += nthr) {
         const int phase = u >= n_up;
         const int tiles = phase ? a.tiles_down : a.tiles_up;

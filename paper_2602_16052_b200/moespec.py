@@ -240,7 +240,7 @@ class Layer:
         _check(lib().moespec_get_stats(self._h, C.byref(st)), "moespec_get_stats")
         return st.as_dict()
 
-    KERNEL_NAMES_TC = ("router_topk", "route", "gather", "ffn", "combine")
+    KERNEL_NAMES_TC = ("router_topk", "route", "gather", "ffn")
     KERNEL_NAMES_CC = ("router_topk", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
 
     def set_profiling(self, on: bool):

@@ -247,7 +247,7 @@ def test_residual_and_host_entry_point():
     o_host = torch.empty_like(h_host).pin_memory()
     layer.verify_layer_host(h_host, 8, 32, o_host)
     assert torch.equal(dev, o_host)
-    assert layer.last_launch_count() >= 5
+    assert layer.last_launch_count() == 4        # router+softmax+top-k, routing, gather, FFN+combine
     layer.destroy()
 
 
