@@ -69,7 +69,8 @@ struct TcArgs {
   int *unit_counter;    // dispenser
   int *ready;           // per (expert, token chunk): finished gate/up units
   int tiles_up;         // gate/up units per chunk = value of ready[] that releases its down units
-  int ru;               // weight rows per unit: 128, 64 or 32
+  int ru;               // weight rows per gate/up unit: 128, 64 or 32
+  int ru_down;          // weight rows per down unit
   int kchunks_up;       // d / 64: K chunks of a gate/up unit
   int kchunks_down;     // f / 64: K chunks of a down unit
   int n_stages;
@@ -195,7 +196,7 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
 // slabs in a gate/up unit) and the 16 KB token region (n_pad rows per chunk), a power of two that
 // divides the unit's chunk count.  Producer, MMA issuer and epilogue all derive it from the unit.
 __device__ __forceinline__ int chunks_per_stage(const TcArgs &a, int phase, int n_pad) {
-  const int cap_a = kARegion / ((phase == 0 ? 2 : 1) * a.ru * 128);
+  const int cap_a = phase == 0 ? kARegion / (2 * a.ru * 128) : kARegion / (a.ru_down * 128);
   const int cap_b = a.b_region / (n_pad * 128);
   const int cap = cap_a < cap_b ? cap_a : cap_b;
   const int kch = phase == 0 ? a.kchunks_up : a.kchunks_down;
@@ -312,11 +313,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int cps = chunks_per_stage(a, phase, n_pad);
       const int k_iters = (phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
       const uint32_t slab_bytes = (uint32_t)n_pad * 128u;           // one K chunk of the unit's token rows
-      const uint32_t sub_bytes = (uint32_t)a.ru * 128u;            // one K chunk of one weight slab
+      const int ru = phase == 0 ? a.ru : a.ru_down;
+      const uint32_t sub_bytes = (uint32_t)ru * 128u;              // one K chunk of one weight slab
       const int w_boxes = (phase == 0 ? 2 : 1) * cps;              // weight copies per stage
-      const int t_per = n_pad / kTokBox;                           // 32-row token copies per K chunk
+      // Token rows arrive in as few copies as possible (the copy engine handles ~13 M boxes/s per SM,
+      // so 8+ boxes per stage would cap the stream): one 128- or 64-row box when n_pad allows, else 32s.
+      const int bsel = n_pad == 128 ? 2 : (n_pad % 64 == 0 ? 1 : 0);
+      const int box_rows = kTokBox << bsel;
+      const int t_per = n_pad / box_rows;                          // token copies per K chunk
       const int n_tok_rows = n_pad;                                // rows that arrive per K chunk
-      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm : &maps.h_mid;
+      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel];
       const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_tok_rows * 128u;
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
@@ -334,12 +340,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           const int j = phase == 0 ? (lane >> 1) : lane;
           const int col = (kc * cps + j) * kChunkK;
           const CUtensorMap *mw = phase == 0 ? ((lane & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
-          tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * a.ru, expert, wpol);
+          tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * ru, expert, wpol);
         }
         for (int tb = lane; tb < cps * t_per; tb += 32) {
           const int j = tb / t_per, r = tb - j * t_per;
           const int col = (kc * cps + j) * kChunkK;
-          tma_load_2d(stage + kARegion + j * slab_bytes + r * (kTokBox * 128), map_b, full, col, row0 + r * kTokBox);
+          tma_load_2d(stage + kARegion + j * slab_bytes + r * (box_rows * 128), map_b, full, col, row0 + r * box_rows);
         }
       }
       if (!ok) break;
@@ -377,7 +383,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // which stages are released.  Descriptors are therefore advanced by adding to the 16-byte-granular
       // address field instead of being rebuilt: +2 per K step of 16 elements, +sub16 per weight slab,
       // +slab16 per token slab.
-      const uint64_t sub16 = (uint64_t)(a.ru * 128 >> 4), slab16 = (uint64_t)(n_pad * 128 >> 4);
+      const uint64_t sub16 = (uint64_t)((un.phase == 0 ? a.ru : a.ru_down) * 128 >> 4), slab16 = (uint64_t)(n_pad * 128 >> 4);
       const uint32_t tmem_u = tmem_d + (uint32_t)n_pad;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
@@ -431,8 +437,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       tc_fence_after();
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
-      const int col_out = un.tile * a.ru + row_in_tile;     // index along f (gate/up) or d (down)
-      const int n_live = quarter * 32 < a.ru ? un.n_rows : 0;   // accumulator lanes beyond RU hold nothing
+      const int ru = un.phase == 0 ? a.ru : a.ru_down;
+      const int col_out = un.tile * ru + row_in_tile;       // index along f (gate/up) or d (down)
+      const int n_live = quarter * 32 < ru ? un.n_rows : 0;     // accumulator lanes beyond the slab hold nothing
       for (int c0 = 0; c0 < n_live; c0 += 16) {
         uint32_t g[16];
         tc_ld16(taddr + c0, g);
@@ -566,10 +573,10 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   };
-  auto rows2d = [&](CUtensorMap *m, void *base, int K) -> CUresult {
+  auto rows2d = [&](CUtensorMap *m, void *base, int K, int box_rows) -> CUresult {
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)R_cap};
     cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    cuuint32_t box[2] = {kChunkK, kTokBox};
+    cuuint32_t box[2] = {kChunkK, (cuuint32_t)box_rows};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   };
@@ -580,8 +587,10 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
     if ((r = weights(&maps->w_up[i], d.w_up, d.f, d.d, box_rows)) != CUDA_SUCCESS) break;
     r = weights(&maps->w_down[i], d.w_down, d.d, d.f, box_rows);
   }
-  if (r == CUDA_SUCCESS) r = rows2d(&maps->x_perm, ws.x_perm, d.d);
-  if (r == CUDA_SUCCESS) r = rows2d(&maps->h_mid, ws.h_mid, d.f);
+  for (int i = 0; i < 3 && r == CUDA_SUCCESS; ++i) {
+    if ((r = rows2d(&maps->x_perm[i], ws.x_perm, d.d, kTokBox << i)) != CUDA_SUCCESS) break;
+    r = rows2d(&maps->h_mid[i], ws.h_mid, d.f, kTokBox << i);
+  }
   if (r != CUDA_SUCCESS) {
     *cu_result = (int)r;
     return cudaErrorInvalidValue;
@@ -613,12 +622,22 @@ int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
   return (long long)active * (D.f / kTile) * 2 < sm_count_cached(D.device) ? 64 : kTile;
 }
 
+// Down units use 128-row slabs: half-height ones would shorten the tail of the list but double the copies
+// per stage, and measured 10 % slower overall.
+int tc_rows_per_down_unit(int ru) {
+  static const int forced = [] { const char *v = getenv("MOESPEC_FORCE_RU_DOWN"); return v ? atoi(v) : 0; }();
+  if (forced == 128 || forced == 64 || forced == 32) return forced;     // experiments only
+  (void)ru;
+  return kTile;
+}
+
 cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
   const int ru = c.ru;
   const int ri = ru == 128 ? 0 : ru == 64 ? 1 : 2;
   TcArgs a;
   a.ru = ru;
+  a.ru_down = tc_rows_per_down_unit(ru);
   a.kchunks_up = D.d / kChunkK;
   a.kchunks_down = D.f / kChunkK;
   const int n_pad_max = c.M >= kMaxTokChunk ? kMaxTokChunk : (c.M + kTokBox - 1) / kTokBox * kTokBox;
@@ -648,9 +667,11 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   TcMapsCall m;
   m.w_gate = maps->w_gate[ri];
   m.w_up = maps->w_up[ri];
-  m.w_down = maps->w_down[ri];
-  m.x_perm = maps->x_perm;
-  m.h_mid = maps->h_mid;
+  m.w_down = maps->w_down[a.ru_down == 128 ? 0 : a.ru_down == 64 ? 1 : 2];
+  for (int i = 0; i < 3; ++i) {
+    m.x_perm[i] = maps->x_perm[i];
+    m.h_mid[i] = maps->h_mid[i];
+  }
   const int grid = sm_count_cached(D.device);
   const size_t smem = (size_t)a.n_stages * a.stage_bytes + kMmaTail + 1024 + kCtrlBytes;
   return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, m, a);

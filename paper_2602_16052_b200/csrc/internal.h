@@ -111,12 +111,15 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down
 // ffn_tc.cu
 struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 32
-  CUtensorMap w_gate[3], w_up[3], w_down[3], x_perm, h_mid;
+  CUtensorMap w_gate[3], w_up[3], w_down[3];
+  CUtensorMap x_perm[3], h_mid[3];   // token-row boxes of 32, 64 and 128 rows
 };
-struct TcMapsCall {        // per launch: the maps of the chosen slab height
-  CUtensorMap w_gate, w_up, w_down, x_perm, h_mid;
+struct TcMapsCall {        // per launch: the weight maps of the chosen slab heights
+  CUtensorMap w_gate, w_up, w_down;
+  CUtensorMap x_perm[3], h_mid[3];
 };
-int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // slab height for a call
+int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // gate/up slab height for a call
+int tc_rows_per_down_unit(int ru);                                         // down slab height for a call
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes

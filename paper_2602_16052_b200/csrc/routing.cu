@@ -654,7 +654,7 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.M = c.M; a.N = D.n_experts; a.k = c.k; a.B = c.B;
   a.policy = D.policy; a.shortlist = D.shortlist; a.renormalize = D.renormalize;
   a.tiles_up = c.ru > 0 ? D.f / c.ru : 0;
-  a.tiles_down = c.ru > 0 ? D.d / c.ru : 0;
+  a.tiles_down = c.ru > 0 ? D.d / tc_rows_per_down_unit(c.ru) : 0;
   a.expert_bytes = 3LL * D.d * D.f * (D.dtype == MOESPEC_BF16 ? 2 : 4);
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
