@@ -202,6 +202,16 @@ int moespec_get_intermediate(moespec_layer_t *layer, int which, void *host_buf, 
 /* Statistics of the last call.  Synchronises the device. */
 int moespec_get_stats(moespec_layer_t *layer, moespec_stats *stats);
 
+/* Test hook for the bounded device-side waits (no fault, trap or hang is involved).
+ * limit_cycles > 0 replaces the default bound (about one second of SM cycles) of every
+ * wait in the expert-FFN kernel; ready_bias > 0 makes every down-projection unit wait
+ * for that many extra gate/up slabs, which are never reported.  With both set, the
+ * waits run out after limit_cycles: each CTA raises its abort flag, lets its copies
+ * land, frees tensor memory and returns; `out` is then undefined and the next
+ * moespec_get_stats reports status = MOESPEC_ERR_TIMEOUT.  Calling with (0, 0) restores
+ * normal operation; the next verify call works as usual. */
+int moespec_debug_set_wait(moespec_layer_t *layer, long long limit_cycles, int ready_bias);
+
 /* Per-kernel timing.  With profiling on, verify calls record a CUDA event on the
  * stream before the first kernel and after every kernel (do not enable it while
  * the stream is being captured into a graph).  get_kernel_times waits for the

@@ -32,6 +32,8 @@ struct moespec_layer {
   const void *hg_in;
   void *hg_out;
   bool graph_usable;
+  long long debug_spin_limit;
+  int debug_ready_bias;
 };
 
 namespace {
@@ -152,6 +154,8 @@ bool is_pinned(const void *p) {
 int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
   if (L->use_tc) c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
+  c.debug_spin_limit = L->debug_spin_limit;
+  c.debug_ready_bias = L->debug_ready_bias;
   int launches = 0;
   cudaError_t e;
   // with profiling on, an event is recorded before the first kernel and after every kernel
@@ -262,6 +266,8 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
     }
   }
   L->profiling = false;
+  L->debug_spin_limit = 0;
+  L->debug_ready_bias = 0;
   L->host_exec = nullptr;
   L->graph_usable = cudaStreamCreateWithFlags(&L->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming) == cudaSuccess;
@@ -456,6 +462,18 @@ int moespec_get_stats(moespec_layer_t *L, moespec_stats *stats) {
   e = cudaMemcpy(&status, L->ws.status, sizeof(int), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return cuda_fail(e);
   stats->status = status;
+  return MOESPEC_OK;
+}
+
+int moespec_debug_set_wait(moespec_layer_t *L, long long limit_cycles, int ready_bias) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (limit_cycles < 0 || ready_bias < 0) return MOESPEC_ERR_INVALID_ARG;
+  L->debug_spin_limit = limit_cycles;
+  L->debug_ready_bias = ready_bias;
+  if (L->host_exec) {            // a captured graph has the old values baked in
+    cudaGraphExecDestroy(L->host_exec);
+    L->host_exec = nullptr;
+  }
   return MOESPEC_OK;
 }
 

@@ -59,7 +59,7 @@ constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
 constexpr int kCtrlBytes = 512;                  // barriers, unit queue, TMEM base, abort flag
 constexpr uint32_t kTmemCols = 512;
-constexpr long long kSpinLimitCycles = 2000000000LL;   // ~1 s at 2 GHz
+constexpr long long kSpinLimitCycles = 2000000000LL;   // default bound of every wait: ~1 s at 2 GHz
 
 constexpr int kQueue = 4;                        // units in flight between the producer and its consumers
 
@@ -87,6 +87,7 @@ struct TcArgs {
   const void *hidden;   // [M, d] bf16 (residual input)
   void *out;            // [M, d] bf16 or fp32
   int M, k, residual, out_is_fp32;
+  long long spin_limit; // cycles after which any wait gives up
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -113,14 +114,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting or the limit expired.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit = kSpinLimitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try(bar, parity)) return true;
     if ((i & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kSpinLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         return false;
       }
@@ -286,7 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       int u_next = n_total;
       if (lane == 0) {
         const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
-        if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag)) ok = 0;
+        if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
         if (ok) {
           q_unit[q] = un;
           mbar_arrive(bar_q_full + 8 * q);          // release: the queue slot is visible to the consumers
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             // the rows of h_mid this unit reads are complete once every gate/up slab of the chunk is done
             const long long t0 = clock64();
             while (ld_acquire(a.ready + un.chunk) < a.tiles_up) {
-              if (*abort_flag || clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; ok = 0; break; }
+              if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
               __nanosleep(64);
             }
             fence_proxy_async();                    // order the acquire before the TMA reads of h_mid
@@ -331,7 +333,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
         if (lane == 0) {
           if (kc == draw_at) u_next = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
-          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) ok = 0;
+          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
           else mbar_expect_tx(full, tx);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -358,7 +360,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       for (uint32_t j = lo; j < it; ++j) {
         const long long t0 = clock64();
         while (!mbar_try(bar_full + 8 * (j % n_stages), (j / n_stages) & 1u))
-          if (clock64() - t0 > kSpinLimitCycles) break;
+          if (clock64() - t0 > a.spin_limit) break;
       }
     }
   } else if (warp == 1 && lane == 0) {
@@ -367,14 +369,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     bool ok = true;
     while (ok) {
       const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
-      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag)) break;
+      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag, a.spin_limit)) break;
       const Unit un = q_unit[q];
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t idesc = instr_desc_bf16(n_pad);
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-      if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag)) break;
+      if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag, a.spin_limit)) break;
       tc_fence_after();
       const uint32_t tmem_d = tmem_base + ab * 256u;
       const int cps = chunks_per_stage(a, un.phase, n_pad);
@@ -387,7 +389,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const uint32_t tmem_u = tmem_d + (uint32_t)n_pad;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
-        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag, a.spin_limit)) { ok = false; break; }
         tc_fence_after();
         uint64_t ad = smem_desc_sw128(smem_base + s * (uint32_t)a.stage_bytes);
         uint64_t bd = ad + (uint64_t)(kARegion >> 4);
@@ -428,12 +430,12 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     uint32_t acc_it = 0, qi = 0;
     while (true) {
       const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
-      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag)) break;
+      if (!mbar_wait(bar_q_full + 8 * q, qph, abort_flag, a.spin_limit)) break;
       const Unit un = q_unit[q];
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag)) break;
+      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag, a.spin_limit)) break;
       tc_fence_after();
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
@@ -489,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     const int n_down = a.n_units[1];
     const long long t0 = clock64();
     while (ld_acquire(a.down_done) < n_down) {
-      if (clock64() - t0 > kSpinLimitCycles) { *abort_flag = 1; break; }
+      if (clock64() - t0 > a.spin_limit) { *abort_flag = 1; break; }
       __nanosleep(128);
     }
   }
@@ -650,7 +652,8 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.n_units = c.ws->counters + 3;
   a.unit_counter = c.ws->unit_counter;
   a.ready = c.ws->ready;
-  a.tiles_up = D.f / ru;
+  a.tiles_up = D.f / ru + c.debug_ready_bias;
+  a.spin_limit = c.debug_spin_limit > 0 ? c.debug_spin_limit : kSpinLimitCycles;
   a.h_mid = reinterpret_cast<__nv_bfloat16 *>(c.ws->h_mid);
   a.y = c.ws->y;
   a.f = D.f;

@@ -71,6 +71,8 @@ struct LaunchCtx {
   int R_cap;            // max_M * max_k
   cudaStream_t stream;
   int ru;               // weight rows per tensor-core work unit for this call (0: CUDA-core path)
+  long long debug_spin_limit = 0;   // test hook: bound of device-side waits in cycles (0 = default)
+  int debug_ready_bias = 0;         // test hook: extra slabs every down unit waits for (never reported)
 };
 
 // Programmatic dependent launch.  Every kernel of the layer is launched with

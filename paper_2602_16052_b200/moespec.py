@@ -29,7 +29,7 @@ ROUTE_STATIC_MAX_M, ROUTE_STATIC_MAX_N, ROUTE_STATIC_MAX_K, ROUTE_STATIC_MAX_ROW
 EXPORTS = [
     "moespec_layer_create", "moespec_verify_layer", "moespec_verify_layer_host",
     "moespec_route_from_logits", "moespec_route_static", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
-    "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
+    "moespec_debug_set_wait", "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
     "moespec_version",
 ]
 
@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.moespec_get_logits.argtypes = [vp, vp]
         L.moespec_get_intermediate.argtypes = [vp, ci, vp, C.c_longlong]
         L.moespec_get_stats.argtypes = [vp, C.POINTER(Stats)]
+        L.moespec_debug_set_wait.argtypes = [vp, C.c_longlong, ci]
         L.moespec_set_profiling.argtypes = [vp, ci]
         L.moespec_get_kernel_times.argtypes = [vp, vp, ci, vp]
         L.moespec_last_launch_count.argtypes = [vp]
@@ -242,6 +243,10 @@ class Layer:
 
     KERNEL_NAMES_TC = ("router_topk", "route", "gather", "ffn")
     KERNEL_NAMES_CC = ("router_topk", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
+
+    def debug_set_wait(self, limit_cycles: int, ready_bias: int):
+        """Test hook: bound of the device-side waits and a ready-counter bias that makes them run out."""
+        _check(lib().moespec_debug_set_wait(self._h, limit_cycles, ready_bias), "moespec_debug_set_wait")
 
     def set_profiling(self, on: bool):
         _check(lib().moespec_set_profiling(self._h, int(on)), "moespec_set_profiling")

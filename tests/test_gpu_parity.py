@@ -319,3 +319,53 @@ def test_stack_teacher_forced_parity_and_drift():
         layer.destroy()
     drift = np.abs(H.f64(x_gpu) - x_ref).max() / np.sqrt(np.mean(x_ref ** 2))
     assert drift < 0.25, f"free-running drift {drift:.3f}"
+
+
+# ------------------------------------------------------------------ bounded waits (no fault involved)
+def test_bounded_wait_expires_cleanly_and_layer_recovers():
+    """Down units are made to wait for slabs that nothing reports; the wait bound is set to ~1 ms.  The
+    kernel must give up, report MOESPEC_ERR_TIMEOUT through the status word and leave the context
+    usable; the next normal call on the same handle must be correct."""
+    m = ms()
+    cfg = synth.CONFIGS["olmoe"].with_(f=256, n_experts=16)
+    case = H.make_case(cfg, 31, seed=12)
+    layer = make_layer(case, 31, cfg.k, out_dtype=torch.float32)
+    good = layer.verify_layer(case["hidden"], cfg.k, 12).clone()
+    assert layer.get_stats()["status"] == 0
+    layer.debug_set_wait(2_000_000, 1)                 # ~1 ms of cycles; one slab too many
+    layer.verify_layer(case["hidden"], cfg.k, 12)
+    torch.cuda.synchronize()                           # returns: nothing hangs, nothing faults
+    assert layer.get_stats()["status"] == m.ERR_TIMEOUT
+    layer.debug_set_wait(0, 0)
+    again = layer.verify_layer(case["hidden"], cfg.k, 12)
+    torch.cuda.synchronize()
+    assert layer.get_stats()["status"] == 0
+    assert torch.equal(good, again)
+    layer.destroy()
+
+
+# ------------------------------------------------------------------ full Mixtral-shaped layer, sampled tokens
+def test_mixtral_full_shape_sampled_tokens():
+    """d=4096, f=14336, N=8, k=2 at full size.  Routing is checked for every token; layer outputs are
+    checked for sampled tokens, whose experts the oracle evaluates one at a time."""
+    m = ms()
+    cfg = synth.CONFIGS["mixtral"]
+    M, B = 15, 4
+    case = H.make_case(cfg, M, seed=5)
+    layer = make_layer(case, M, cfg.k, out_dtype=torch.float32)
+    out = layer.verify_layer(case["hidden"], cfg.k, B)
+    torch.cuda.synchronize()
+    assert layer.get_stats()["status"] == 0
+    r = H.oracle_route(layer.get_logits(), cfg.k, B, orc.SUBSTITUTION, orc.FROM_ALL, True)
+    H.compare_routing(layer.get_routing(), r, orc.SUBSTITUTION, cfg.k)
+    sample = [0, 7, 14]
+    Hs = H.f64(case["hidden"][sample])
+    ref = np.zeros((len(sample), cfg.d))
+    for e in sorted({i for t in sample for i in r["assign"][t]}):
+        y = orc.expert_ffn(Hs, H.f64(case["w_gate"][e]), H.f64(case["w_up"][e]), H.f64(case["w_down"][e]))
+        for j, t in enumerate(sample):
+            ref[j] += r["wgt"][t, e] * y[j]
+    o = H.f64(out[sample])
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    assert np.max(np.abs(o - ref)) <= BF16_TOL * rms
+    layer.destroy()
