@@ -234,7 +234,13 @@ def run_tables(args, device):
                 act = sum(s_["n_active"] for s_ in st) / len(st)
                 uni = sum(s_["n_union"] for s_ in st) / len(st)
                 by = algorithmic_bytes(cfg, M, act, 2 if out_dtype == torch.bfloat16 else 4)
+                cpu_us = None
+                if args.tables_cpu:        # the oracle on one layer of this point, once (host cores)
+                    case = oracle_case(cfg, M, seed=2000, device=device)
+                    cpu_us, cpu_cores, _ = time_oracle(cfg, M, B, 0.0, 1, case)
+                    del case
                 print(json.dumps({"table": name, "layers": L, "M": M, "B": B, "us_per_layer": round(us, 2),
+                                  "cpu_oracle_us": None if cpu_us is None else round(cpu_us),
                                   "n_active": round(act, 2), "n_union": round(uni, 2), "MB": round(by / 1e6, 1),
                                   "GBs": round(by / us / 1e3, 1), "frac_of_" + peak_kind: round(by / us / 1e3 / peak, 3),
                                   "ideal_us": round(by / peak / 1e3, 1)}), flush=True)
@@ -258,10 +264,11 @@ def job_us_per_layer(job_ms: float, steps: int, world: int) -> float:
     return job_ms * 1e3 / (steps * world)
 
 
-def oracle_case(cfg, M, seed):
-    L = synth.gen_layer(cfg, seed=seed, layer=0, device="cpu")
-    h = synth.gen_hidden(cfg, M, seed=seed, layer=0, device="cpu")
-    f64 = lambda t: t.to(torch.float64).numpy()
+def oracle_case(cfg, M, seed, device="cpu"):
+    """Inputs of one layer as fp64 numpy arrays (generated on `device`: the generator gives the same bits)."""
+    L = synth.gen_layer(cfg, seed=seed, layer=0, device=device)
+    h = synth.gen_hidden(cfg, M, seed=seed, layer=0, device=device)
+    f64 = lambda t: t.to("cpu").to(torch.float64).numpy()
     return {k: f64(v) for k, v in L.items()}, f64(h)
 
 
@@ -319,6 +326,8 @@ def main():
     ap.add_argument("--copies", type=int, default=N_COPIES, help="independently seeded layer copies rotated over")
     ap.add_argument("--tables", default="", help="comma-separated workload names (tiny is excluded): sweep M and B "
                     "of each and print one JSON line per point instead of the benchmark line")
+    ap.add_argument("--tables-cpu", action="store_true",
+                    help="with --tables: also time the CPU oracle once per point (one layer, host cores)")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed steps (for profiler captures); prints a short line")
     args = ap.parse_args()
