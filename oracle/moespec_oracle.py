@@ -21,6 +21,7 @@ Steps (notation of the paper: M tokens h_t, N experts, top-k, budget B):
       over the original top-k; raw or renormalised per architecture          Section 2.1, Section 3.3
   O8  out_t = sum_{i in A(t)} wgt[t,i] * E_i(h_t), E_i a bias-free SwiGLU FFN Eq. 2 / 7 / 8
   O9  canonical per-expert gather order of routed (token, expert) pairs      Appendix C
+  O10 static ranking: calibration counts c_i and the fixed ordering          Eq. 4
 
 Readings of points the paper leaves open (tie-breaks, candidate set of the
 shortlist, expert form, router bias) are listed in the repository's design
@@ -42,6 +43,7 @@ SUBSTITUTION = 1   # Eq. 8
 TRUNCATION = 2     # Eq. 7
 FROM_ALL = 1       # Algorithm 1 literal: all N experts compete for the shortlist
 FROM_UNION = 2     # only experts of the union E(D) compete (Section 3.1 framing)
+STATIC = 3         # fixed ordering from calibration counts (Eq. 4, "Static Ranking")
 
 
 # --------------------------------------------------------------------------- O1
@@ -122,6 +124,17 @@ def shortlist(s, B, candidates):
     """
     cand = list(candidates)
     return _ranked(s, cand)[:max(0, min(B, len(cand)))]
+
+
+def static_counts(z_calib, k):
+    """c_i = number of calibration tokens whose natural top-k contains expert i (Eq. 4)."""
+    T, _, natcnt = natural_topk(z_calib, k)
+    return natcnt
+
+
+def static_ranking(counts):
+    """Experts ordered by (selection count descending, index ascending): the fixed ordering of Eq. 4."""
+    return _ranked(counts, range(len(counts)))
 
 
 # --------------------------------------------------------------------------- O6
@@ -234,15 +247,22 @@ def canonical_permutation(A, N):
 
 
 # ------------------------------------------------------------------ whole layer
-def route(z, k, B, policy, shortlist_mode, renormalize):
-    """Steps O2..O7 and O9 from fp32 logits.  Returns a dict of every stage."""
+def route(z, k, B, policy, shortlist_mode, renormalize, static_rank=None):
+    """Steps O2..O7 and O9 from fp32 logits.  Returns a dict of every stage.
+
+    With shortlist_mode STATIC the shortlist is the first B experts of `static_rank`
+    (Section 3.2, "Static Ranking": the B experts with the highest calibration count);
+    the router-based scores are still reported but do not choose S."""
     z = np.asarray(z, dtype=np.float32)
     M, N = z.shape
     p = softmax_rows(z)
     T, union, natcnt = natural_topk(z, k)
     s = router_scores(p)
-    cand = range(N) if shortlist_mode == FROM_ALL else union
-    S = shortlist(s, min(B, N), cand)
+    if shortlist_mode == STATIC:
+        S = list(static_rank)[:max(0, min(B, len(static_rank)))]
+    else:
+        cand = range(N) if shortlist_mode == FROM_ALL else union
+        S = shortlist(s, min(B, N), cand)
     A = assign(z, S, T, k, policy)
     Wt = gate_weights(p, A, T, policy, renormalize)
     count, offset, active, perm, row_of = canonical_permutation(A, N)
@@ -253,10 +273,10 @@ def route(z, k, B, policy, shortlist_mode, renormalize):
 
 
 def verify_layer(H, router_w, router_bias, w_gate, w_up, w_down, k, B, policy, shortlist_mode,
-                 renormalize, logits=None, expert_rows=None):
+                 renormalize, logits=None, expert_rows=None, static_rank=None):
     """Algorithm 1 end to end.  `logits` (fp32 [M,N]) replaces step O1 when given."""
     z = router_logits(H, router_w, router_bias) if logits is None else np.asarray(logits, dtype=np.float32)
-    r = route(z, k, B, policy, shortlist_mode, renormalize)
+    r = route(z, k, B, policy, shortlist_mode, renormalize, static_rank)
     r["out"] = layer_output(H, r["wgt"], w_gate, w_up, w_down, expert_rows)
     return r
 

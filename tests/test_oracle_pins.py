@@ -374,3 +374,48 @@ def test_round_bf16_matches_torch():
     x[:4] = [0.0, 1.00390625, 1.01171875, -3.0e-39]               # ties to even both ways, a denormal
     ref = torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16).double().numpy()
     np.testing.assert_array_equal(orc.round_bf16(x), ref)
+
+
+# ------------------------------------------------------------ O10 static ranking (Eq. 4)
+def test_static_counts_brute_force_and_ranking():
+    rng = np.random.default_rng(8)
+    z = rng.integers(-3, 4, size=(57, 9)).astype(np.float32)        # ties included
+    k = 3
+    c = orc.static_counts(z, k)
+    # brute force: expert i is in T_k(h) iff fewer than k experts rank strictly before it
+    want = [0] * 9
+    for t in range(z.shape[0]):
+        for i in range(9):
+            if sum(beats(z[t], j, i) for j in range(9)) < k:
+                want[i] += 1
+    assert c == want and sum(c) == z.shape[0] * k
+    rank = orc.static_ranking(c)
+    assert sorted(rank) == list(range(9))
+    assert all(c[a] > c[b] or (c[a] == c[b] and a < b) for a, b in zip(rank, rank[1:]))
+    # counts do not depend on the order of the calibration tokens, and add over calibration chunks
+    perm = rng.permutation(z.shape[0])
+    assert orc.static_counts(z[perm], k) == c
+    c2 = [a + b for a, b in zip(orc.static_counts(z[:20], k), orc.static_counts(z[20:], k))]
+    assert c2 == c
+
+
+def test_static_shortlist_is_the_prefix_of_the_fixed_ordering():
+    cfg, H, L = tiny_inputs()
+    z = orc.router_logits(H, L["router_w"], L["router_bias"])
+    rank = orc.static_ranking(orc.static_counts(z, cfg.k))
+    for B in (1, 4, 8, 16, 30):
+        for pol in (orc.SUBSTITUTION, orc.TRUNCATION):
+            r = orc.route(z, cfg.k, B, pol, orc.STATIC, True, static_rank=rank)
+            assert r["S"] == rank[:min(B, cfg.n_experts)]
+            S = set(r["S"])
+            for t in range(H.shape[0]):
+                Tk = set(r["topk"][t])
+                if pol == orc.TRUNCATION:
+                    assert set(r["assign"][t]) == Tk & S
+                else:
+                    assert set(r["assign"][t]) <= S and len(r["assign"][t]) == min(cfg.k, len(S))
+    # a budget of all N experts reproduces the unbudgeted layer whatever the ordering
+    full = run(cfg, H, L, cfg.n_experts)
+    st = orc.verify_layer(H, L["router_w"], L["router_bias"], L["w_gate"], L["w_up"], L["w_down"], cfg.k,
+                          cfg.n_experts, orc.SUBSTITUTION, orc.STATIC, True, static_rank=rank)
+    np.testing.assert_array_equal(st["out"], full["out"])
