@@ -420,6 +420,28 @@ def main():
             sweep.append({"M": M, "B": Bs, "us": us_b, "n_active": act, "GBs": by / (us_b * 1e-6) / 1e9,
                           "frac": by / (us_b * 1e-6) / 1e9 / peak})
 
+    # static ranking (Eq. 4) on the same workload: fixed ordering from 512 calibration tokens per copy
+    static_line = None
+    if not args.no_sweep:
+        from paper_2602_16052_b200 import moespec
+        st_layers = []
+        for c, L0 in enumerate(layers):
+            rw, rb, wg, wu, wd = L0._keep
+            SL = moespec.Layer(rw, rb, wg, wu, wd, max_M=128, max_k=cfg.k, policy=moespec.SUBSTITUTION,
+                               shortlist=moespec.STATIC, renormalize=True, out_dtype=out_dtype)
+            for j in range(4):
+                SL.calibrate(synth.gen_hidden(cfg, 128, seed=5000 + 10 * c + j, device=device), cfg.k)
+            SL.set_static_ranking()
+            st_layers.append(SL)
+        n_st = max(20, args.steps // 4)
+        ms_st = time_steps(st_layers, hiddens, outs, k, B, n_st, 5, barrier)
+        act = sum(L_.get_stats()["n_active"] for L_ in st_layers) / len(st_layers)
+        cov = sum(L_.get_stats()["coverage"] for L_ in st_layers) / len(st_layers)
+        static_line = {"M": M, "B": B, "us": ms_st * 1e3 / n_st, "n_active": act, "coverage": cov,
+                       "calibration_tokens": 512}
+        for SL in st_layers:
+            SL.destroy()
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         us, cores, reps = time_oracle(cfg, M, B, 10.0, 6)
@@ -443,6 +465,7 @@ def main():
             "roofline": roofline,
             "cpu_baseline": cpu,
             "sweep": sweep,
+            "static_ranking": static_line,
         }
         print(json.dumps(line), flush=True)
     for L in layers:

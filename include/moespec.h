@@ -57,7 +57,10 @@ typedef enum { MOESPEC_SUBSTITUTION = 1, MOESPEC_TRUNCATION = 2 } moespec_policy
  * (all N experts ranked by s_i, so |S| = min(B, N)).  FROM_UNION restricts the
  * candidates to the union E(D) of Eq. 3 (so |S| = min(B, |E|) and any
  * B >= |E| reproduces the unbudgeted layer). */
-typedef enum { MOESPEC_FROM_ALL = 1, MOESPEC_FROM_UNION = 2 } moespec_shortlist_t;
+/* MOESPEC_STATIC: the "Static Ranking" of Section 3.2.  The shortlist is the first B
+ * experts of a fixed ordering by calibration count c_i (Eq. 4), set with
+ * moespec_calibrate / moespec_set_static_ranking; it does not depend on the tree. */
+typedef enum { MOESPEC_FROM_ALL = 1, MOESPEC_FROM_UNION = 2, MOESPEC_STATIC = 3 } moespec_shortlist_t;
 /* Expert-FFN kernel choice.  AUTO picks the tensor-core kernel for bf16 and the
  * CUDA-core kernel for fp32 (fp32 accuracy needs full-precision FMAs). */
 typedef enum { MOESPEC_FFN_AUTO = 0, MOESPEC_FFN_CUDA_CORE = 1, MOESPEC_FFN_TENSOR_CORE = 2 } moespec_ffn_t;
@@ -118,6 +121,21 @@ int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int 
  * first.  Pageable buffers take a plain copy-launch-copy path on `stream`. */
 int moespec_verify_layer_host(moespec_layer_t *layer, const void *hidden_host, int M, int k, int B,
                               void *out_host, void *stream);
+
+/* Static ranking, Eq. 4: c_i = number of calibration tokens whose natural top-k contains
+ * expert i.  moespec_calibrate runs the router, softmax and top-k on hidden (device
+ * [M, d], dtype) and adds each token's top-k to the layer's counters (device, 64-bit);
+ * call it as often as there is calibration data.  It enqueues on `stream` and returns.
+ * moespec_get_static_counts copies c[N] to a HOST buffer (synchronises).
+ * moespec_set_static_ranking fixes the ordering a MOESPEC_STATIC layer uses: `ranked`
+ * is a HOST array of n distinct expert ids, best first; NULL means "order the experts
+ * by (c_i descending, index ascending)" (synchronises to read the counters).  A verify
+ * call on a MOESPEC_STATIC layer without a ranking returns INVALID_ARG.
+ * moespec_reset_calibration zeroes the counters. */
+int moespec_calibrate(moespec_layer_t *layer, const void *hidden, int M, int k, void *stream);
+int moespec_get_static_counts(moespec_layer_t *layer, long long *counts_host);
+int moespec_set_static_ranking(moespec_layer_t *layer, const int *ranked_host, int n);
+int moespec_reset_calibration(moespec_layer_t *layer);
 
 /* Steps after the router projection only (softmax, top-k, Eq. 5 scores,
  * shortlist, Eq. 7 / Eq. 8 re-routing, Appendix C gather order), from caller-

@@ -117,6 +117,9 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.colmask, N * (size_t)w.mask_words);
   c.take(w.arrive, M);
   c.take(w.arrive_route, 4);
+  c.take(w.calib_count, N);
+  c.take(w.static_pos, N);
+  w.n_static = 0;
   c.take(w.units, max_chunks * (tiles_up + tiles_down));
   c.take(w.ready, max_chunks);
   c.take(w.unit_counter, 4);
@@ -134,6 +137,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
 
 int validate_call(moespec_layer *L, int M, int k, int B) {
   const moespec_layer_desc &d = L->desc;
+  if (d.shortlist == MOESPEC_STATIC && L->ws.n_static == 0) return MOESPEC_ERR_INVALID_ARG;   // no ranking set
   if (M < 0 || M > d.max_M) return MOESPEC_ERR_INVALID_ARG;
   if (k < 1 || k > d.max_k || k > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
   if (B < 1) return MOESPEC_ERR_INVALID_ARG;
@@ -209,7 +213,8 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   if (d.out_dtype != 0 && d.out_dtype != MOESPEC_BF16 && d.out_dtype != MOESPEC_FP32) return MOESPEC_ERR_INVALID_ARG;
   if (d.dtype == MOESPEC_FP32 && d.out_dtype == MOESPEC_BF16) return MOESPEC_ERR_UNSUPPORTED;
   if (d.policy != MOESPEC_SUBSTITUTION && d.policy != MOESPEC_TRUNCATION) return MOESPEC_ERR_INVALID_ARG;
-  if (d.shortlist != MOESPEC_FROM_ALL && d.shortlist != MOESPEC_FROM_UNION) return MOESPEC_ERR_INVALID_ARG;
+  if (d.shortlist != MOESPEC_FROM_ALL && d.shortlist != MOESPEC_FROM_UNION && d.shortlist != MOESPEC_STATIC)
+    return MOESPEC_ERR_INVALID_ARG;
   if ((d.renormalize | 1) != 1 || (d.residual | 1) != 1) return MOESPEC_ERR_INVALID_ARG;
   if (d.ffn_kernel < MOESPEC_FFN_AUTO || d.ffn_kernel > MOESPEC_FFN_TENSOR_CORE) return MOESPEC_ERR_INVALID_ARG;
   if (d.d < 64 || d.f < 64 || d.n_experts < 1 || d.max_M < 1 || d.max_k < 1 || d.device < 0)
@@ -367,6 +372,97 @@ int moespec_verify_layer_host(moespec_layer_t *L, const void *hidden_host, int M
   return MOESPEC_OK;
 }
 
+#define MOESPEC_COPY_BACK(dst, src, count)                                                         \
+  do {                                                                                             \
+    if ((dst) && (count) > 0) {                                                                    \
+      cudaError_t e_ = cudaMemcpy((dst), (src), sizeof(*(dst)) * (size_t)(count), cudaMemcpyDeviceToHost); \
+      if (e_ != cudaSuccess) return cuda_fail(e_);                                                 \
+    }                                                                                              \
+  } while (0)
+
+int moespec_calibrate(moespec_layer_t *L, const void *hidden, int M, int k, void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  const moespec_layer_desc &d = L->desc;
+  if (M < 0 || M > d.max_M || k < 1 || k > d.max_k || k > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (M == 0) return MOESPEC_OK;
+  if (!hidden) return MOESPEC_ERR_NULL_POINTER;
+  if (!aligned16(hidden)) return MOESPEC_ERR_UNSUPPORTED;
+  DeviceGuard guard(d.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  LaunchCtx c{&L->desc, &L->ws, M, k, 1, L->R_cap, static_cast<cudaStream_t>(stream), 0};
+  cudaError_t e = launch_router_logits(c, hidden);
+  if (e == cudaSuccess) e = launch_calib_accumulate(c);
+  if (e != cudaSuccess) return cuda_fail(e);
+  L->last_M = M;
+  L->last_k = k;
+  L->last_launches = 2;
+  return MOESPEC_OK;
+}
+
+int moespec_get_static_counts(moespec_layer_t *L, long long *counts_host) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!counts_host) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  MOESPEC_COPY_BACK(counts_host, L->ws.calib_count, L->desc.n_experts);
+  return MOESPEC_OK;
+}
+
+int moespec_reset_calibration(moespec_layer_t *L) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemset(L->ws.calib_count, 0, sizeof(long long) * L->desc.n_experts);
+  return e == cudaSuccess ? MOESPEC_OK : cuda_fail(e);
+}
+
+int moespec_set_static_ranking(moespec_layer_t *L, const int *ranked_host, int n) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  const int N = L->desc.n_experts;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  std::vector<int> order;
+  if (ranked_host) {
+    if (n < 1 || n > N) return MOESPEC_ERR_INVALID_ARG;
+    order.assign(ranked_host, ranked_host + n);
+  } else {
+    std::vector<long long> cnt(N);
+    e = cudaMemcpy(cnt.data(), L->ws.calib_count, sizeof(long long) * N, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    order.resize(N);
+    for (int i = 0; i < N; ++i) order[i] = i;
+    // (count descending, expert index ascending); insertion sort keeps the file free of <algorithm> lambdas
+    for (int i = 1; i < N; ++i) {
+      const int x = order[i];
+      int j = i - 1;
+      while (j >= 0 && (cnt[order[j]] < cnt[x] || (cnt[order[j]] == cnt[x] && order[j] > x))) {
+        order[j + 1] = order[j];
+        --j;
+      }
+      order[j + 1] = x;
+    }
+  }
+  std::vector<int> pos(N, 0x7fffffff);
+  for (size_t r = 0; r < order.size(); ++r) {
+    const int ex = order[r];
+    if (ex < 0 || ex >= N || pos[ex] != 0x7fffffff) return MOESPEC_ERR_INVALID_ARG;   // out of range or repeated
+    pos[ex] = (int)r;
+  }
+  e = cudaMemcpy(L->ws.static_pos, pos.data(), sizeof(int) * N, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e);
+  L->ws.n_static = (int)order.size();
+  if (L->host_exec) {            // a captured graph has the old ordering size baked into its arguments
+    cudaGraphExecDestroy(L->host_exec);
+    L->host_exec = nullptr;
+  }
+  return MOESPEC_OK;
+}
+
 int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, int k, int B, void *stream) {
   if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
   int rc = validate_call(L, M, k, B);
@@ -386,13 +482,6 @@ int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, in
   return MOESPEC_OK;
 }
 
-#define MOESPEC_COPY_BACK(dst, src, count)                                                         \
-  do {                                                                                             \
-    if ((dst) && (count) > 0) {                                                                    \
-      cudaError_t e_ = cudaMemcpy((dst), (src), sizeof(*(dst)) * (size_t)(count), cudaMemcpyDeviceToHost); \
-      if (e_ != cudaSuccess) return cuda_fail(e_);                                                 \
-    }                                                                                              \
-  } while (0)
 
 int moespec_get_routing(moespec_layer_t *L, int *S_rank, int *n_S, int *topk_idx, int *assign_idx, float *gate_w,
                         int *count, int *offset, int *perm_row2tok, int *tokslot2row, double *score,

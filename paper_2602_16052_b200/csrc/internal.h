@@ -51,6 +51,9 @@ struct Workspace {
   int *arrive;          // [max_M] arrival counters of router_topk_kernel's token tiles
   int *arrive_route;    // [1] arrival counter of route_kernel's CTAs
   int mask_words;       // ceil(max_M / 32)
+  long long *calib_count;   // [N] Eq. 4 calibration counts c_i
+  int *static_pos;          // [N] position of expert i in the fixed ordering (INT_MAX: not listed)
+  int n_static;             // experts in the fixed ordering (0: none set)
   Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
   int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
   int *unit_counter;    // [0] next unit to hand out, [1] finished down units; zeroed by the route kernel
@@ -108,6 +111,7 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden);
 cudaError_t launch_route(const LaunchCtx &c, const float *logits);   // softmax/top-k kernel + route kernel
 cudaError_t launch_route_after_router(const LaunchCtx &c);           // route kernel only
+cudaError_t launch_calib_accumulate(const LaunchCtx &c);             // c_i += natural counts of the last router launch
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
 // ffn_simple.cu
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down

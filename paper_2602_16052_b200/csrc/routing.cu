@@ -442,8 +442,22 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   const int n_union = __syncthreads_count(in_union);
   ROUTE_MARK();
   const int n_cand = __syncthreads_count(tid < N && s_cand[tid]);
-  const int nS = min(a.B, n_cand);
-  {
+  const bool fixed = a.shortlist == MOESPEC_STATIC;
+  const int nS = fixed ? min(a.B, ws.n_static) : min(a.B, n_cand);
+  if (fixed) {
+    // static ranking (Eq. 4): the shortlist is the first nS experts of the fixed ordering
+    bool in_S = false;
+    if (tid < N) {
+      const int pos = ws.static_pos[tid];
+      in_S = pos < nS;
+      if (in_S) {
+        s_Srank[pos] = tid;
+        if (blockIdx.x == 0) ws.S_rank[pos] = tid;
+      }
+    }
+    const unsigned word = __ballot_sync(kFull, in_S);
+    if (lane == 0) s_Smask[warp] = word;
+  } else {
     // one thread per expert; every thread walks the same j, so the shared-memory reads are broadcasts
     // Branch-free rank by counting.  s_score holds score+1 for candidates and 0 for the others, so a
     // non-candidate never outranks a candidate.
@@ -661,6 +675,24 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);
   if (a.N <= 128) return launch_kernel(route_kernel<4>, grid, block, 0, c.stream, a);
   return launch_kernel(route_kernel<8>, grid, block, 0, c.stream, a);
+}
+
+// Eq. 4: add the natural top-k counts of the last router launch to the calibration counters and
+// clear the per-call accumulators (no routing kernel follows a calibration pass).
+__global__ void __launch_bounds__(256) calib_accumulate_kernel(long long *calib, int *natcnt, unsigned long long *score_fx,
+                                                               int N) {
+  pdl_trigger();
+  pdl_wait();
+  for (int i = threadIdx.x; i < N; i += blockDim.x) {
+    calib[i] += natcnt[i];
+    natcnt[i] = 0;
+    score_fx[i] = 0ull;
+  }
+}
+
+cudaError_t launch_calib_accumulate(const LaunchCtx &c) {
+  return launch_kernel(calib_accumulate_kernel, dim3(1), dim3(256), 0, c.stream, c.ws->calib_count, c.ws->natcnt_acc,
+                       c.ws->score_fx, c.desc->n_experts);
 }
 
 // Routing after router_topk_kernel has filled logits, prob, topk_idx and the score accumulators.

@@ -18,7 +18,7 @@ LIB_PATH = os.environ.get("MOESPEC_LIB") or os.path.join(_HERE, "libmoespec.so")
 
 BF16, FP32 = 1, 2
 SUBSTITUTION, TRUNCATION = 1, 2
-FROM_ALL, FROM_UNION = 1, 2
+FROM_ALL, FROM_UNION, STATIC = 1, 2, 3
 FFN_AUTO, FFN_CUDA_CORE, FFN_TENSOR_CORE = 0, 1, 2
 
 OK = 0
@@ -28,6 +28,7 @@ ROUTE_STATIC_MAX_M, ROUTE_STATIC_MAX_N, ROUTE_STATIC_MAX_K, ROUTE_STATIC_MAX_ROW
 
 EXPORTS = [
     "moespec_layer_create", "moespec_verify_layer", "moespec_verify_layer_host",
+    "moespec_calibrate", "moespec_get_static_counts", "moespec_set_static_ranking", "moespec_reset_calibration",
     "moespec_route_from_logits", "moespec_route_static", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
     "moespec_debug_set_wait", "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
     "moespec_version",
@@ -76,6 +77,10 @@ def lib() -> C.CDLL:
         L.moespec_layer_create.argtypes = [C.POINTER(LayerDesc), C.POINTER(vp)]
         L.moespec_verify_layer.argtypes = [vp, vp, ci, ci, ci, vp, vp]
         L.moespec_verify_layer_host.argtypes = [vp, vp, ci, ci, ci, vp, vp]
+        L.moespec_calibrate.argtypes = [vp, vp, ci, ci, vp]
+        L.moespec_get_static_counts.argtypes = [vp, vp]
+        L.moespec_set_static_ranking.argtypes = [vp, vp, ci]
+        L.moespec_reset_calibration.argtypes = [vp]
         L.moespec_route_from_logits.argtypes = [vp, vp, ci, ci, ci, vp]
         L.moespec_route_static.argtypes = [vp] + [ci] * 7 + [vp] * 11
         L.moespec_get_routing.argtypes = [vp] + [vp] * 11
@@ -191,6 +196,27 @@ class Layer:
                                                _stream_ptr(stream)), "moespec_verify_layer_host")
         self._last = (M, k)
         return out_host
+
+    # -- static ranking (Eq. 4)
+    def calibrate(self, hidden: torch.Tensor, k: int, stream=None):
+        M = hidden.shape[0]
+        _check(lib().moespec_calibrate(self._h, hidden.data_ptr(), M, k, _stream_ptr(stream)), "moespec_calibrate")
+        self._last = (M, k)
+
+    def get_static_counts(self) -> np.ndarray:
+        c = np.zeros(self.N, dtype=np.int64)
+        _check(lib().moespec_get_static_counts(self._h, _np_ptr(c)), "moespec_get_static_counts")
+        return c
+
+    def set_static_ranking(self, ranked=None):
+        if ranked is None:
+            _check(lib().moespec_set_static_ranking(self._h, None, 0), "moespec_set_static_ranking")
+        else:
+            a = np.ascontiguousarray(ranked, dtype=np.int32)
+            _check(lib().moespec_set_static_ranking(self._h, _np_ptr(a), len(a)), "moespec_set_static_ranking")
+
+    def reset_calibration(self):
+        _check(lib().moespec_reset_calibration(self._h), "moespec_reset_calibration")
 
     def route_from_logits(self, logits: torch.Tensor, k: int, B: int, stream=None):
         M = logits.shape[0]

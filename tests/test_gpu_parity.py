@@ -369,3 +369,49 @@ def test_mixtral_full_shape_sampled_tokens():
     rms = float(np.sqrt(np.mean(ref ** 2)))
     assert np.max(np.abs(o - ref)) <= BF16_TOL * rms
     layer.destroy()
+
+
+# ------------------------------------------------------------------ static ranking (Eq. 4)
+def test_static_ranking_calibration_and_layer():
+    """Calibration counts are exact integers (compared with the oracle's count on the GPU's own
+    logits, chunk by chunk); a MOESPEC_STATIC layer then keeps the first B experts of the fixed
+    ordering whatever the tree looks like."""
+    m = ms()
+    cfg = synth.CONFIGS["olmoe"].with_(f=256)
+    case = H.make_case(cfg, 63, seed=14)
+    layer = make_layer(case, 128, cfg.k, shortlist=m.STATIC, out_dtype=torch.float32)
+    with pytest.raises(m.MoeSpecError):                      # no ranking yet
+        layer.verify_layer(case["hidden"], cfg.k, 16)
+    want = np.zeros(cfg.n_experts, dtype=np.int64)
+    for chunk, Mc in enumerate((128, 77, 1)):                # ragged calibration chunks
+        hc = synth.gen_hidden(cfg, Mc, seed=100 + chunk, device="cuda")
+        layer.calibrate(hc, cfg.k)
+        want += np.array(orc.static_counts(layer.get_logits(), cfg.k), dtype=np.int64)
+    got = layer.get_static_counts()
+    assert np.array_equal(got, want) and got.sum() == (128 + 77 + 1) * cfg.k
+    layer.set_static_ranking()                               # order by (count desc, index asc)
+    rank = orc.static_ranking(want.tolist())
+    for B, policy in ((16, m.SUBSTITUTION), (32, m.SUBSTITUTION), (64, m.SUBSTITUTION)):
+        out = layer.verify_layer(case["hidden"], cfg.k, B)
+        torch.cuda.synchronize()
+        r = orc.verify_layer(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]),
+                             H.LazyF64(case["w_gate"]), H.LazyF64(case["w_up"]), H.LazyF64(case["w_down"]), cfg.k, B,
+                             policy, orc.STATIC, True, logits=layer.get_logits(), static_rank=rank)
+        assert r["S"] == rank[:B]
+        H.compare_routing(layer.get_routing(), r, policy, cfg.k)
+        check_out(out, r["out"], cfg.dtype)
+    # an explicit ordering, truncation policy
+    layer.destroy()
+    layer = make_layer(case, 63, cfg.k, shortlist=m.STATIC, policy=m.TRUNCATION, out_dtype=torch.float32)
+    explicit = list(range(cfg.n_experts - 1, -1, -1))[:20]
+    layer.set_static_ranking(explicit)
+    out = layer.verify_layer(case["hidden"], cfg.k, 12)
+    torch.cuda.synchronize()
+    r = orc.verify_layer(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]),
+                         H.LazyF64(case["w_gate"]), H.LazyF64(case["w_up"]), H.LazyF64(case["w_down"]), cfg.k, 12,
+                         orc.TRUNCATION, orc.STATIC, True, logits=layer.get_logits(), static_rank=explicit)
+    H.compare_routing(layer.get_routing(), r, orc.TRUNCATION, cfg.k)
+    check_out(out, r["out"], cfg.dtype)
+    with pytest.raises(m.MoeSpecError):
+        layer.set_static_ranking([3, 3, 5])                  # repeated expert
+    layer.destroy()
