@@ -420,6 +420,28 @@ def main():
             sweep.append({"M": M, "B": Bs, "us": us_b, "n_active": act, "GBs": by / (us_b * 1e-6) / 1e9,
                           "frac": by / (us_b * 1e-6) / 1e9 / peak})
 
+    # time against kept experts: slope = FFN stream per expert, intercept = routing chain + FFN ramp and tail
+    fit = None
+    if len(sweep) >= 3:
+        xs = np.array([p_["n_active"] for p_ in sweep]); ys = np.array([p_["us"] for p_ in sweep])
+        slope, icpt = np.polyfit(xs, ys, 1)
+        fit = {"us_per_expert": float(slope), "intercept_us": float(icpt),
+               "marginal_GBs": cfg.expert_weight_bytes() / (float(slope) * 1e-6) / 1e9 if slope > 0 else None}
+
+    # read-only stream rate of this GPU (a library reduction over 2 GiB), context for the copy-based peak
+    big = torch.empty(1 << 30, dtype=torch.bfloat16, device=device).fill_(1)
+    for _ in range(2):
+        big.sum()
+    torch.cuda.synchronize()
+    r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    r0.record()
+    for _ in range(5):
+        big.sum()
+    r1.record()
+    torch.cuda.synchronize()
+    read_stream_gbs = 5 * big.numel() * 2 / (r0.elapsed_time(r1) * 1e-3) / 1e9
+    del big
+
     # static ranking (Eq. 4) on the same workload: fixed ordering from 512 calibration tokens per copy
     static_line = None
     if not args.no_sweep:
@@ -466,6 +488,8 @@ def main():
             "cpu_baseline": cpu,
             "sweep": sweep,
             "static_ranking": static_line,
+            "fit_time_vs_active_experts": fit,
+            "read_stream_GBs_torch_sum": read_stream_gbs,
         }
         print(json.dumps(line), flush=True)
     for L in layers:
