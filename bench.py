@@ -75,7 +75,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -318,7 +318,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="moespec", choices=["moespec", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -405,6 +405,9 @@ def main():
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
         "traffic": FFN_DRAM_TRAFFIC_BYTES,
         "algorithmic_bytes_per_layer": ffn_bytes, "kernel_us": {n: v * 1e3 for n, v in kt.items()},
+        # share of the event-bracketed kernel time spent choosing experts (router, shortlist, re-routing,
+        # gather); the paper quotes 2-3 % of whole-model generation time for its selection step
+        "selection_share_of_layer": (sum(v for n, v in kt.items() if n != "ffn") / sum(kt.values())),
         "whole_layer": {"bytes": layer_bytes, "GBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9,
                         "frac": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / peak,
                         "frac_of_nominal_8TBs": layer_bytes / (us_per_layer * world * 1e-6) / 1e9 / 8000.0},
@@ -419,6 +422,21 @@ def main():
             by = algorithmic_bytes(cfg, M, act, 4)
             sweep.append({"M": M, "B": Bs, "us": us_b, "n_active": act, "GBs": by / (us_b * 1e-6) / 1e9,
                           "frac": by / (us_b * 1e-6) / 1e9 / peak})
+
+    # raw (non-renormalised) mixing weights, the other architecture choice of Section 2.1: same kernels
+    raw_line = None
+    if not args.no_sweep:
+        from paper_2602_16052_b200 import moespec as _m
+        raw_layers = []
+        for L0 in layers:
+            rw, rb, wg, wu, wd = L0._keep
+            raw_layers.append(_m.Layer(rw, rb, wg, wu, wd, max_M=M, max_k=cfg.k, policy=_m.SUBSTITUTION,
+                                       shortlist=_m.FROM_ALL, renormalize=False, out_dtype=out_dtype))
+        n_raw = max(20, args.steps // 4)
+        ms_raw = time_steps(raw_layers, hiddens, outs, k, B, n_raw, 5, barrier)
+        raw_line = {"M": M, "B": B, "us": ms_raw * 1e3 / n_raw, "renormalize": False}
+        for RL in raw_layers:
+            RL.destroy()
 
     # time against kept experts: slope = FFN stream per expert, intercept = routing chain + FFN ramp and tail
     fit = None
@@ -488,6 +506,7 @@ def main():
             "cpu_baseline": cpu,
             "sweep": sweep,
             "static_ranking": static_line,
+            "raw_gating": raw_line,
             "fit_time_vs_active_experts": fit,
             "read_stream_GBs_torch_sum": read_stream_gbs,
         }
