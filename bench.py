@@ -120,7 +120,7 @@ class ClockSampler:
 
 def algorithmic_bytes(cfg, M, n_active, out_bytes):
     """Bytes the method itself must move for one layer: kept experts' weights, the router, hidden in, out."""
-    w = 2 if cfg.dtype == "bf16" else 4
+    w = 4 if cfg.dtype == "fp32" else 2
     return n_active * 3 * cfg.d * cfg.f * w + cfg.n_experts * cfg.d * w + M * cfg.d * w + M * cfg.d * out_bytes
 
 

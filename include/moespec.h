@@ -50,7 +50,8 @@ typedef enum {
   MOESPEC_ERR_TOO_LARGE = -9      /* a size exceeds the fixed capacity of moespec_route_static   */
 } moespec_status;
 
-typedef enum { MOESPEC_BF16 = 1, MOESPEC_FP32 = 2 } moespec_dtype_t;
+/* MOESPEC_FP16 is the paper's own precision (Appendix A, "All models use FP16 precision"). */
+typedef enum { MOESPEC_BF16 = 1, MOESPEC_FP32 = 2, MOESPEC_FP16 = 3 } moespec_dtype_t;
 /* Token policy of Section 3.3: Eq. 8 / Eq. 7. */
 typedef enum { MOESPEC_SUBSTITUTION = 1, MOESPEC_TRUNCATION = 2 } moespec_policy_t;
 /* Which experts compete for the shortlist.  FROM_ALL is Algorithm 1 as printed
@@ -62,7 +63,7 @@ typedef enum { MOESPEC_SUBSTITUTION = 1, MOESPEC_TRUNCATION = 2 } moespec_policy
  * moespec_calibrate / moespec_set_static_ranking; it does not depend on the tree. */
 typedef enum { MOESPEC_FROM_ALL = 1, MOESPEC_FROM_UNION = 2, MOESPEC_STATIC = 3 } moespec_shortlist_t;
 /* Expert-FFN kernel choice.  AUTO picks the tensor-core kernel for bf16 and the
- * CUDA-core kernel for fp32 (fp32 accuracy needs full-precision FMAs). */
+ * CUDA-core kernel for fp32 (fp32 accuracy needs full-precision FMAs); fp16 is treated like bf16. */
 typedef enum { MOESPEC_FFN_AUTO = 0, MOESPEC_FFN_CUDA_CORE = 1, MOESPEC_FFN_TENSOR_CORE = 2 } moespec_ffn_t;
 
 typedef struct {
@@ -72,8 +73,8 @@ typedef struct {
   int max_M;          /* largest M any call will pass (sizes the workspace), 1..4096              */
   int max_k;          /* largest k any call will pass, 1..min(N, 32)                              */
   int dtype;          /* moespec_dtype_t of weights and hidden; accumulation is always fp32       */
-  int out_dtype;      /* moespec_dtype_t of out; 0 = same as dtype.  MOESPEC_FP32 with bf16 weights
-                         returns the fp32 accumulators unrounded                                  */
+  int out_dtype;      /* moespec_dtype_t of out; 0 = same as dtype.  MOESPEC_FP32 with 16-bit weights
+                         returns the fp32 accumulators unrounded; other mixes are unsupported    */
   int policy;         /* moespec_policy_t; 0 is invalid: the caller must choose                   */
   int shortlist;      /* moespec_shortlist_t; 0 is invalid: the caller must choose                */
   int renormalize;    /* 1: mixing weights are renormalised (Section 2.1, "OLMoE renormalizes"); 0: raw g_i */

@@ -70,8 +70,8 @@ struct DeviceGuard {
   }
 };
 
-size_t elt_bytes(const moespec_layer_desc &d) { return d.dtype == MOESPEC_BF16 ? 2 : 4; }
-size_t out_elt_bytes(const moespec_layer_desc &d) { return (d.out_dtype ? d.out_dtype : d.dtype) == MOESPEC_BF16 ? 2 : 4; }
+size_t elt_bytes(const moespec_layer_desc &d) { return dtype_bytes(d.dtype); }
+size_t out_elt_bytes(const moespec_layer_desc &d) { return dtype_bytes(d.out_dtype ? d.out_dtype : d.dtype); }
 
 struct Carver {
   size_t off = 0;
@@ -209,9 +209,11 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   if (!desc || !out_layer) return MOESPEC_ERR_NULL_POINTER;
   const moespec_layer_desc &d = *desc;
   if (!d.router_w || !d.w_gate || !d.w_up || !d.w_down) return MOESPEC_ERR_NULL_POINTER;
-  if (d.dtype != MOESPEC_BF16 && d.dtype != MOESPEC_FP32) return MOESPEC_ERR_INVALID_ARG;
-  if (d.out_dtype != 0 && d.out_dtype != MOESPEC_BF16 && d.out_dtype != MOESPEC_FP32) return MOESPEC_ERR_INVALID_ARG;
-  if (d.dtype == MOESPEC_FP32 && d.out_dtype == MOESPEC_BF16) return MOESPEC_ERR_UNSUPPORTED;
+  if (d.dtype != MOESPEC_BF16 && d.dtype != MOESPEC_FP32 && d.dtype != MOESPEC_FP16) return MOESPEC_ERR_INVALID_ARG;
+  if (d.out_dtype != 0 && d.out_dtype != MOESPEC_BF16 && d.out_dtype != MOESPEC_FP32 && d.out_dtype != MOESPEC_FP16)
+    return MOESPEC_ERR_INVALID_ARG;
+  // out is either the layer's dtype or fp32
+  if (d.out_dtype != 0 && d.out_dtype != d.dtype && d.out_dtype != MOESPEC_FP32) return MOESPEC_ERR_UNSUPPORTED;
   if (d.policy != MOESPEC_SUBSTITUTION && d.policy != MOESPEC_TRUNCATION) return MOESPEC_ERR_INVALID_ARG;
   if (d.shortlist != MOESPEC_FROM_ALL && d.shortlist != MOESPEC_FROM_UNION && d.shortlist != MOESPEC_STATIC)
     return MOESPEC_ERR_INVALID_ARG;
@@ -226,8 +228,8 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   if (!aligned16(d.router_w) || !aligned16(d.w_gate) || !aligned16(d.w_up) || !aligned16(d.w_down))
     return MOESPEC_ERR_UNSUPPORTED;
   bool use_tc = d.ffn_kernel == MOESPEC_FFN_TENSOR_CORE ||
-                (d.ffn_kernel == MOESPEC_FFN_AUTO && d.dtype == MOESPEC_BF16);
-  if (use_tc && (d.dtype != MOESPEC_BF16 || d.d % kTile || d.f % kTile)) {
+                (d.ffn_kernel == MOESPEC_FFN_AUTO && is_16bit(d.dtype));
+  if (use_tc && (!is_16bit(d.dtype) || d.d % kTile || d.f % kTile)) {
     if (d.ffn_kernel == MOESPEC_FFN_TENSOR_CORE) return MOESPEC_ERR_UNSUPPORTED;
     use_tc = false;
   }

@@ -14,6 +14,12 @@ __device__ __forceinline__ float4 load4(const __nv_bfloat16 *p) {
   float2 a = __bfloat1622float2(h[0]), b = __bfloat1622float2(h[1]);
   return make_float4(a.x, a.y, b.x, b.y);
 }
+__device__ __forceinline__ float4 load4(const __half *p) {
+  uint2 raw = *reinterpret_cast<const uint2 *>(p);
+  const __half2 *h = reinterpret_cast<const __half2 *>(&raw);
+  float2 a = __half22float2(h[0]), b = __half22float2(h[1]);
+  return make_float4(a.x, a.y, b.x, b.y);
+}
 __device__ __forceinline__ void store4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
 __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
   __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
@@ -25,6 +31,14 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *p, float4 v) {
 
 // Grid (M, ceil(d / 1024)): one float4 of one token per thread.  The up-to-k rows of y are all
 // loaded before the first FMA (one memory round trip), then added in slot order.
+__device__ __forceinline__ void store4(__half *p, float4 v) {
+  __half2 lo = __floats2half2_rn(v.x, v.y), hi = __floats2half2_rn(v.z, v.w);
+  uint2 raw;
+  raw.x = *reinterpret_cast<uint32_t *>(&lo);
+  raw.y = *reinterpret_cast<uint32_t *>(&hi);
+  *reinterpret_cast<uint2 *>(p) = raw;
+}
+
 template <typename T, typename TO>
 __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ y,
                                                       const float *__restrict__ gate_w,
@@ -82,6 +96,8 @@ cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out) {
   const int od = D.out_dtype ? D.out_dtype : D.dtype;
   if (D.dtype == MOESPEC_BF16 && od == MOESPEC_BF16) return launch_t<__nv_bfloat16, __nv_bfloat16>(c, hidden, out);
   if (D.dtype == MOESPEC_BF16) return launch_t<__nv_bfloat16, float>(c, hidden, out);
+  if (D.dtype == MOESPEC_FP16 && od == MOESPEC_FP16) return launch_t<__half, __half>(c, hidden, out);
+  if (D.dtype == MOESPEC_FP16) return launch_t<__half, float>(c, hidden, out);
   return launch_t<float, float>(c, hidden, out);
 }
 

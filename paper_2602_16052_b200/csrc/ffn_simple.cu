@@ -8,8 +8,10 @@ namespace moespec {
 
 __device__ __forceinline__ float cc_to_float(float v) { return v; }
 __device__ __forceinline__ float cc_to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float cc_to_float(__half v) { return __half2float(v); }
 __device__ __forceinline__ void cc_store(float *p, float v) { *p = v; }
 __device__ __forceinline__ void cc_store(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+__device__ __forceinline__ void cc_store(__half *p, float v) { *p = __float2half_rn(v); }
 
 constexpr int kColsPerBlock = 64;
 
@@ -109,7 +111,9 @@ static cudaError_t launch_cc(const LaunchCtx &c, int phase) {
 }
 
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase) {
-  return c.desc->dtype == MOESPEC_BF16 ? launch_cc<__nv_bfloat16>(c, phase) : launch_cc<float>(c, phase);
+  if (c.desc->dtype == MOESPEC_BF16) return launch_cc<__nv_bfloat16>(c, phase);
+  if (c.desc->dtype == MOESPEC_FP16) return launch_cc<__half>(c, phase);
+  return launch_cc<float>(c, phase);
 }
 
 }  // namespace moespec

@@ -1,4 +1,4 @@
-// Tensor-core expert FFN for bf16: the weight-streaming kernel of the layer.
+// Tensor-core expert FFN for bf16 and fp16: the weight-streaming kernel of the layer.
 //
 // Work unit = one slab of RU (128, 64 or 32) rows of one kept expert's weight
 // matrix against one chunk (<= 128) of that expert's routed rows.  RU is chosen
@@ -76,7 +76,8 @@ struct TcArgs {
   int n_stages;
   int b_region;         // token-row bytes per stage
   int stage_bytes;      // kARegion + b_region
-  __nv_bfloat16 *h_mid; // [R, f]
+  void *h_mid;          // [R, f] bf16 or fp16
+  int is_fp16;          // 16-bit format of weights, hidden and h_mid: 0 bf16, 1 fp16
   float *y;             // [R, d]
   int f, d;
   int *status;
@@ -187,9 +188,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
   d |= (uint64_t)2 << 61;                          // SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16 (format 1) or fp16 (format 0), both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_16bit(int n, int is_fp16) {
+  const uint32_t fmt = is_fp16 ? 0u : 1u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
 }
 
 }  // namespace
@@ -374,7 +376,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
-      const uint32_t idesc = instr_desc_bf16(n_pad);
+      const uint32_t idesc = instr_desc_16bit(n_pad, a.is_fp16);
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
       if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag, a.spin_limit)) break;
       tc_fence_after();
@@ -454,7 +456,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             if (c0 + i < un.n_rows) {
               const float gv = __uint_as_float(g[i]), uv = __uint_as_float(up[i]);
               const float m = gv / (1.f + __expf(-gv)) * uv;
-              a.h_mid[(size_t)(un.row0 + c0 + i) * a.f + col_out] = __float2bfloat16_rn(m);
+              const size_t off = (size_t)(un.row0 + c0 + i) * a.f + col_out;
+              if (a.is_fp16) reinterpret_cast<__half *>(a.h_mid)[off] = __float2half_rn(m);
+              else reinterpret_cast<__nv_bfloat16 *>(a.h_mid)[off] = __float2bfloat16_rn(m);
             }
           }
         } else {
@@ -528,20 +532,32 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         }
       }
       if (a.residual) {
-        const uint2 raw = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(a.hidden) +
+        const uint2 raw = *reinterpret_cast<const uint2 *>(reinterpret_cast<const uint16_t *>(a.hidden) +
                                                             (size_t)t * d + c);
-        const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
-        const float2 lo = __bfloat1622float2(h2[0]), hi = __bfloat1622float2(h2[1]);
+        float2 lo, hi;
+        if (a.is_fp16) {
+          const __half2 *h2 = reinterpret_cast<const __half2 *>(&raw);
+          lo = __half22float2(h2[0]); hi = __half22float2(h2[1]);
+        } else {
+          const __nv_bfloat162 *h2 = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+          lo = __bfloat1622float2(h2[0]); hi = __bfloat1622float2(h2[1]);
+        }
         acc.x += lo.x; acc.y += lo.y; acc.z += hi.x; acc.w += hi.y;
       }
       if (a.out_is_fp32) {
         *reinterpret_cast<float4 *>(reinterpret_cast<float *>(a.out) + (size_t)t * d + c) = acc;
       } else {
-        __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
         uint2 raw;
-        raw.x = *reinterpret_cast<uint32_t *>(&lo);
-        raw.y = *reinterpret_cast<uint32_t *>(&hi);
-        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.out) + (size_t)t * d + c) = raw;
+        if (a.is_fp16) {
+          __half2 lo = __floats2half2_rn(acc.x, acc.y), hi = __floats2half2_rn(acc.z, acc.w);
+          raw.x = *reinterpret_cast<uint32_t *>(&lo);
+          raw.y = *reinterpret_cast<uint32_t *>(&hi);
+        } else {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x, acc.y), hi = __floats2bfloat162_rn(acc.z, acc.w);
+          raw.x = *reinterpret_cast<uint32_t *>(&lo);
+          raw.y = *reinterpret_cast<uint32_t *>(&hi);
+        }
+        *reinterpret_cast<uint2 *>(reinterpret_cast<uint16_t *>(a.out) + (size_t)t * d + c) = raw;
       }
     }
   }
@@ -567,11 +583,13 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
   cudaError_t e = get_encode_fn(&enc);
   if (e != cudaSuccess) return e;
   const cuuint32_t ones[3] = {1, 1, 1};
+  const CUtensorMapDataType tm_dtype =
+      d.dtype == MOESPEC_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   auto weights = [&](CUtensorMap *m, const void *base, int rows, int K, int box_rows) -> CUresult {
     cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)d.n_experts};
     cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)rows * K * 2};
     cuuint32_t box[3] = {kChunkK, (cuuint32_t)box_rows, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, ones,
+    return enc(m, tm_dtype, 3, const_cast<void *>(base), dims, strides, box, ones,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   };
@@ -579,7 +597,7 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)R_cap};
     cuuint64_t strides[1] = {(cuuint64_t)K * 2};
     cuuint32_t box[2] = {kChunkK, (cuuint32_t)box_rows};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    return enc(m, tm_dtype, 2, base, dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   };
   CUresult r = CUDA_SUCCESS;
@@ -654,7 +672,8 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.ready = c.ws->ready;
   a.tiles_up = D.f / ru + c.debug_ready_bias;
   a.spin_limit = c.debug_spin_limit > 0 ? c.debug_spin_limit : kSpinLimitCycles;
-  a.h_mid = reinterpret_cast<__nv_bfloat16 *>(c.ws->h_mid);
+  a.h_mid = c.ws->h_mid;
+  a.is_fp16 = D.dtype == MOESPEC_FP16;
   a.y = c.ws->y;
   a.f = D.f;
   a.d = D.d;

@@ -3,10 +3,14 @@
 #include <cuda_runtime.h>
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <stdint.h>
 #include "../../include/moespec.h"
 
 namespace moespec {
+
+inline bool is_16bit(int dtype) { return dtype == MOESPEC_BF16 || dtype == MOESPEC_FP16; }
+inline int dtype_bytes(int dtype) { return is_16bit(dtype) ? 2 : 4; }
 
 constexpr int kMaxExperts = 256;           // N limit: 8 experts per lane in the warp-wide rankings
 constexpr int kMaskWords = kMaxExperts / 32;

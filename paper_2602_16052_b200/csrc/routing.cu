@@ -24,6 +24,7 @@ namespace moespec {
 
 __device__ __forceinline__ float to_float(float v) { return v; }
 __device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+__device__ __forceinline__ float to_float(__half v) { return __half2float(v); }
 
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kScoreScale = 4503599627370496.0;   // 2^52: scores are sums of round(p * 2^52)
@@ -258,7 +259,9 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
-  return c.desc->dtype == MOESPEC_BF16 ? launch_router_t<__nv_bfloat16>(c, hidden) : launch_router_t<float>(c, hidden);
+  if (c.desc->dtype == MOESPEC_BF16) return launch_router_t<__nv_bfloat16>(c, hidden);
+  if (c.desc->dtype == MOESPEC_FP16) return launch_router_t<__half>(c, hidden);
+  return launch_router_t<float>(c, hidden);
 }
 
 // Softmax and top-k from caller-supplied logits: one warp per token.
@@ -669,7 +672,7 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.policy = D.policy; a.shortlist = D.shortlist; a.renormalize = D.renormalize;
   a.tiles_up = c.ru > 0 ? D.f / c.ru : 0;
   a.tiles_down = c.ru > 0 ? D.d / tc_rows_per_down_unit(c.ru) : 0;
-  a.expert_bytes = 3LL * D.d * D.f * (D.dtype == MOESPEC_BF16 ? 2 : 4);
+  a.expert_bytes = 3LL * D.d * D.f * dtype_bytes(D.dtype);
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
   if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);
@@ -725,7 +728,7 @@ __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restric
 
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
   const moespec_layer_desc &D = *c.desc;
-  const int row_vec = D.d * (D.dtype == MOESPEC_BF16 ? 2 : 4) / 16;
+  const int row_vec = D.d * dtype_bytes(D.dtype) / 16;
   const int rows = c.M * c.k;
   if (rows == 0) return cudaSuccess;
   return launch_kernel(gather_rows_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,

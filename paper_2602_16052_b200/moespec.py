@@ -16,7 +16,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("MOESPEC_LIB") or os.path.join(_HERE, "libmoespec.so")   # override for debug builds
 
-BF16, FP32 = 1, 2
+BF16, FP32, FP16 = 1, 2, 3
+_DTYPES = {torch.bfloat16: 1, torch.float32: 2, torch.float16: 3}
 SUBSTITUTION, TRUNCATION = 1, 2
 FROM_ALL, FROM_UNION, STATIC = 1, 2, 3
 FFN_AUTO, FFN_CUDA_CORE, FFN_TENSOR_CORE = 0, 1, 2
@@ -160,7 +161,7 @@ class Layer:
         f = w_gate.shape[1]
         if tuple(w_gate.shape) != (N, f, d) or tuple(w_up.shape) != (N, f, d) or tuple(w_down.shape) != (N, d, f):
             raise ValueError("weight shapes must be [N,f,d], [N,f,d], [N,d,f]")
-        dt = {torch.bfloat16: BF16, torch.float32: FP32}[router_w.dtype]
+        dt = _DTYPES[router_w.dtype]
         if router_bias is not None:
             router_bias = router_bias.to(device=router_w.device, dtype=torch.float32).contiguous()
         self._keep = (router_w, router_bias, w_gate, w_up, w_down)
@@ -169,7 +170,7 @@ class Layer:
         self.out_dtype = out_dtype or router_w.dtype
         self.device = router_w.device
         desc = LayerDesc(d=d, n_experts=N, f=f, max_M=max_M, max_k=max_k, dtype=dt,
-                         out_dtype={torch.bfloat16: BF16, torch.float32: FP32}[self.out_dtype], policy=policy,
+                         out_dtype=_DTYPES[self.out_dtype], policy=policy,
                          shortlist=shortlist, renormalize=int(renormalize), residual=int(residual),
                          ffn_kernel=ffn_kernel, device=router_w.device.index or 0,
                          router_w=router_w.data_ptr(),

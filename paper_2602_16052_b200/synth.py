@@ -114,7 +114,7 @@ def normal_fp32(key: int, start: int, count: int, sigma: float, device="cpu") ->
 
 
 def torch_dtype(name: str) -> torch.dtype:
-    return {"bf16": torch.bfloat16, "fp32": torch.float32}[name]
+    return {"bf16": torch.bfloat16, "fp32": torch.float32, "fp16": torch.float16}[name]
 
 
 @dataclass(frozen=True)
@@ -125,7 +125,7 @@ class LayerConfig:
     n_experts: int
     k: int
     f: int
-    dtype: str          # storage dtype of weights, hidden and out: "bf16" | "fp32"
+    dtype: str          # storage dtype of weights, hidden and out: "bf16" | "fp16" | "fp32"
     slope: float        # router bias = -slope * ln(rank)
     n_layers: int = 1
 
@@ -133,7 +133,7 @@ class LayerConfig:
         return replace(self, **kw)
 
     def expert_weight_bytes(self) -> int:
-        w = 2 if self.dtype == "bf16" else 4
+        w = 4 if self.dtype == "fp32" else 2
         return 3 * self.d * self.f * w
 
 

@@ -16,6 +16,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 BF16_TOL = 2e-2
+FP16_TOL = 5e-3     # fp16 keeps 11 significant bits: h_mid rounding is 8x finer than bf16's
 FP32_TOL = 1e-5
 
 
@@ -38,12 +39,14 @@ def check_out(out, ref, dtype):
     live = np.any(ref != 0.0, axis=1)
     assert not np.any(o[~live]), "a token with no kept expert must get exact zeros"
     rms = float(np.sqrt(np.mean(ref[live] ** 2))) if live.any() else 0.0
-    if dtype == "bf16" and out.dtype == torch.float32:
+    if dtype in ("bf16", "fp16") and out.dtype == torch.float32:
+        tol = BF16_TOL if dtype == "bf16" else FP16_TOL
         err = float(np.max(np.abs(o - ref)))
-        assert err <= BF16_TOL * rms, f"max err {err:.3e} > {BF16_TOL} * rms {rms:.3e}"
-    elif dtype == "bf16":
-        # out stored as bf16: the stated bar plus the final rounding of the result itself (half an ulp <= 2^-8 |ref|)
-        bound = BF16_TOL * rms + 2.0 ** -8 * np.abs(ref)
+        assert err <= tol * rms, f"max err {err:.3e} > {tol} * rms {rms:.3e}"
+    elif dtype in ("bf16", "fp16"):
+        # out stored in 16 bits: the bar plus the final rounding of the result itself
+        # (half an ulp <= 2^-8 |ref| for bf16, 2^-11 |ref| for fp16)
+        bound = (BF16_TOL * rms + 2.0 ** -8 * np.abs(ref)) if dtype == "bf16" else (FP16_TOL * rms + 2.0 ** -11 * np.abs(ref))
         assert np.all(np.abs(o - ref) <= bound), f"worst {np.max(np.abs(o - ref) / np.maximum(bound, 1e-300)):.2f}x of bound"
     else:
         bound = FP32_TOL * np.maximum(np.abs(ref), rms)
@@ -415,3 +418,16 @@ def test_static_ranking_calibration_and_layer():
     with pytest.raises(m.MoeSpecError):
         layer.set_static_ranking([3, 3, 5])                  # repeated expert
     layer.destroy()
+
+
+# ------------------------------------------------------------------ fp16, the paper's own precision
+@pytest.mark.parametrize("ffn", ["cuda_core", "tensor_core"])
+def test_fp16_layer(ffn):
+    m = ms()
+    cfg = synth.CONFIGS["olmoe"].with_(dtype="fp16")
+    kern = m.FFN_CUDA_CORE if ffn == "cuda_core" else m.FFN_TENSOR_CORE
+    case = H.make_case(cfg, 63, seed=21)
+    assert case["w_gate"].dtype == torch.float16
+    run_e2e(cfg, 63, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, kern, case=case)
+    run_e2e(cfg, 63, 12, orc.TRUNCATION, orc.FROM_UNION, False, kern, case=case, out_dtype=torch.float16,
+            residual=True)
