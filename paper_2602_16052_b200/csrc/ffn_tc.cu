@@ -444,28 +444,44 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int ru = un.phase == 0 ? a.ru : a.ru_down;
       const int col_out = un.tile * ru + row_in_tile;       // index along f (gate/up) or d (down)
       const int n_live = quarter * 32 < ru ? un.n_rows : 0;     // accumulator lanes beyond the slab hold nothing
-      for (int c0 = 0; c0 < n_live; c0 += 16) {
-        uint32_t g[16];
-        tc_ld16(taddr + c0, g);
-        if (un.phase == 0) {
-          uint32_t up[16];
+      // One warp per scheduler runs this loop, so it is latency-bound: the sixteen columns of a step are
+      // computed as independent chains (approximate exp and divide: two instructions each, error far
+      // below the 16-bit rounding of the result) before the first store is issued.
+      if (un.phase == 0) {
+        for (int c0 = 0; c0 < n_live; c0 += 16) {
+          uint32_t g[16], up[16];
+          tc_ld16(taddr + c0, g);
           tc_ld16(taddr + n_pad + c0, up);
           tc_ld_wait();
+          float m[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            if (c0 + i < un.n_rows) {
-              const float gv = __uint_as_float(g[i]), uv = __uint_as_float(up[i]);
-              const float m = gv / (1.f + __expf(-gv)) * uv;
-              const size_t off = (size_t)(un.row0 + c0 + i) * a.f + col_out;
-              if (a.is_fp16) reinterpret_cast<__half *>(a.h_mid)[off] = __float2half_rn(m);
-              else reinterpret_cast<__nv_bfloat16 *>(a.h_mid)[off] = __float2bfloat16_rn(m);
-            }
+            const float gv = __uint_as_float(g[i]);
+            m[i] = __fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(up[i]);
           }
-        } else {
+          const int n_here = min(16, un.n_rows - c0);
+          if (a.is_fp16) {
+            __half *dst = reinterpret_cast<__half *>(a.h_mid) + (size_t)(un.row0 + c0) * a.f + col_out;
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (i < n_here) dst[(size_t)i * a.f] = __float2half_rn(m[i]);
+          } else {
+            __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(a.h_mid) + (size_t)(un.row0 + c0) * a.f + col_out;
+#pragma unroll
+            for (int i = 0; i < 16; ++i)
+              if (i < n_here) dst[(size_t)i * a.f] = __float2bfloat16_rn(m[i]);
+          }
+        }
+      } else {
+        for (int c0 = 0; c0 < n_live; c0 += 16) {
+          uint32_t g[16];
+          tc_ld16(taddr + c0, g);
           tc_ld_wait();
+          const int n_here = min(16, un.n_rows - c0);
+          float *dst = a.y + (size_t)(un.row0 + c0) * a.d + col_out;
 #pragma unroll
           for (int i = 0; i < 16; ++i)
-            if (c0 + i < un.n_rows) a.y[(size_t)(un.row0 + c0 + i) * a.d + col_out] = __uint_as_float(g[i]);
+            if (i < n_here) dst[(size_t)i * a.d] = __uint_as_float(g[i]);
         }
       }
       tc_fence_before();
