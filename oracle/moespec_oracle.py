@@ -22,6 +22,10 @@ Steps (notation of the paper: M tokens h_t, N experts, top-k, budget B):
   O8  out_t = sum_{i in A(t)} wgt[t,i] * E_i(h_t), E_i a bias-free SwiGLU FFN Eq. 2 / 7 / 8
   O9  canonical per-expert gather order of routed (token, expert) pairs      Appendix C
   O10 static ranking: calibration counts c_i and the fixed ordering          Eq. 4
+  O11 residual stack: x_{l+1} = storage(x_l + layer_l(x_l)), budget B_l per layer
+      (Section 4: the budget is enforced at every MoE layer of the model)
+  O12 oracle ranking: greedy minimisation of the reconstruction error        Eq. 6
+  O13 reconstruction error ||O_S - O*||^2 / ||O*||^2                         Section 4.5
 
 Readings of points the paper leaves open (tie-breaks, candidate set of the
 shortlist, expert form, router bias) are listed in the repository's design
@@ -29,7 +33,10 @@ notes; each function states the one it takes.
 
 Pins: every function here is pinned by tests that do not restate its formula
 (brute force over subsets, invariants, closed forms, reductions to a plain
-top-k MoE / a single SwiGLU FFN / a dense softmax mixture).  The one unpinned
+top-k MoE / a single SwiGLU FFN / a dense softmax mixture / a plain residual
+SwiGLU stack, a hand-worked greedy example, the k = 1 closed form of Eq. 6, and
+the identity between the objective of Eq. 6 and the error of the separately
+pinned truncation layer of Eq. 7).  The one unpinned
 item is statistical: the synthetic router's union sizes and coverage are only
 reported beside the paper's Figure 2 / 4 / 7 numbers, which depend on trained
 weights ("parity unpinned" for those statistics; no oracle output depends on
@@ -293,7 +300,117 @@ def round_bf16(x):
 
 
 def round_storage(x, dtype):
-    """Round to the storage dtype ("bf16" or "fp32") and return fp64."""
+    """Round to the storage dtype ("bf16", "fp16" or "fp32") and return fp64."""
     if dtype == "bf16":
         return round_bf16(x)
+    if dtype == "fp16":
+        return np.asarray(x, dtype=np.float64).astype(np.float16).astype(np.float64)
     return np.asarray(x, dtype=np.float32).astype(np.float64)
+
+
+# -------------------------------------------------------------------------- O11
+def verify_stack(H, layers, k, budgets, policy, shortlist_mode, renormalize, storage, static_ranks=None):
+    """L budgeted MoE layers on a residual stream: x_0 = H, x_{l+1} = storage(x_l + out_l(x_l)).
+
+    The budget is enforced at each MoE layer (abstract; Section 4.6 leaves a
+    per-layer budget open, so `budgets` is one B per layer).  Only the MoE blocks
+    are on this path: attention and normalisation between them are not part of
+    the method.  `layers[l]` is a dict with router_w, router_bias, w_gate, w_up,
+    w_down.  The stream is rounded to the storage dtype after every layer, as a
+    model that keeps activations in that dtype does.  Returns the list
+    [x_0, ..., x_L] and the per-layer routing dicts.
+    """
+    xs = [np.asarray(H, dtype=np.float64)]
+    routes = []
+    for l, Lw in enumerate(layers):
+        r = verify_layer(xs[-1], Lw["router_w"], Lw["router_bias"], Lw["w_gate"], Lw["w_up"], Lw["w_down"], k,
+                         budgets[l], policy, shortlist_mode, renormalize,
+                         static_rank=None if static_ranks is None else static_ranks[l])
+        xs.append(round_storage(xs[-1] + r["out"], storage))
+        routes.append(r)
+    return xs, routes
+
+
+# -------------------------------------------------------------------------- O12
+def expert_contributions(H, z, k, renormalize, w_gate, w_up, w_down):
+    """C[t][i] = g_i(h_t) * E_i(h_t) for i in T_k(h_t): the terms of the gold output O* (Eq. 2, Eq. 6).
+
+    g is the mixing weight of the unpruned model: the softmax probability, divided
+    by the sum over T_k(h_t) when the architecture renormalises (Section 2.1).
+    Returns (T, C) with C a list of dicts expert -> fp64 vector [d].
+    """
+    H = np.asarray(H, dtype=np.float64)
+    z = np.asarray(z, dtype=np.float32)
+    M, N = z.shape
+    p = softmax_rows(z)
+    T, _, _ = natural_topk(z, k)
+    W = gate_weights(p, T, T, TRUNCATION, renormalize)
+    C = [dict() for _ in range(M)]
+    for i in range(N):
+        toks = [t for t in range(M) if i in T[t]]
+        if not toks:
+            continue
+        y = expert_ffn(H[toks], w_gate[i], w_up[i], w_down[i])
+        for row, t in enumerate(toks):
+            C[t][i] = W[t, i] * y[row]
+    return T, C
+
+
+def gold_output(T, C, d):
+    """O*_t = sum_{i in T_k(h_t)} g_i(h_t) E_i(h_t), experts added in ascending index (Eq. 6, first line)."""
+    out = np.zeros((len(T), d), dtype=np.float64)
+    for t in range(len(T)):
+        for i in sorted(T[t]):
+            out[t] += C[t][i]
+    return out
+
+
+def subset_error(T, C, O_star, S):
+    """sum_t || O*_t - sum_{j in S and in T_k(h_t)} g_j(h_t) E_j(h_t) ||^2: the objective of Eq. 6 for the set S.
+
+    Reading: the inner sum runs over the experts of S that the token actually
+    routes to; an expert outside T_k(h_t) has no term in O*_t and contributes
+    nothing for that token (the truncation output with the original weights).
+    """
+    inS = set(S)
+    err = 0.0
+    for t in range(len(T)):
+        approx = np.zeros_like(O_star[t])
+        for j in sorted(T[t]):
+            if j in inS:
+                approx += C[t][j]
+        diff = O_star[t] - approx
+        err += float(diff @ diff)
+    return err
+
+
+def oracle_ranking(T, C, N, d, B):
+    """Greedy ordering of Eq. 6: starting from the empty set, B times add the expert outside S
+    whose addition leaves the smallest objective (ties -> lower expert index).
+
+    Every candidate's objective is evaluated from its definition (no incremental
+    update).  Returns (order, errors) with errors[b] the objective after b+1 picks.
+    """
+    O_star = gold_output(T, C, d)
+    S, errs = [], []
+    for _ in range(min(B, N)):
+        best, best_err = -1, None
+        for i in range(N):
+            if i in S:
+                continue
+            e = subset_error(T, C, O_star, S + [i])
+            if best_err is None or e < best_err:       # strict: the first (lowest) index keeps a tie
+                best, best_err = i, e
+        S.append(best)
+        errs.append(best_err)
+    return S, errs
+
+
+# -------------------------------------------------------------------------- O13
+def reconstruction_error(O_S, O_star):
+    """||O_S - O*||_F^2 / ||O*||_F^2 over all tokens of the tree (Section 4.5)."""
+    O_S = np.asarray(O_S, dtype=np.float64)
+    O_star = np.asarray(O_star, dtype=np.float64)
+    den = float(np.sum(O_star * O_star))
+    num = float(np.sum((O_S - O_star) ** 2))
+    return num / den if den > 0.0 else (0.0 if num == 0.0 else float("inf"))

@@ -155,23 +155,32 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   const int t0 = blockIdx.y * TT;
   const int i = blockIdx.x * 8 + warp;
   __shared__ int s_last;
+  constexpr int VEC = 16 / sizeof(T);
+  constexpr int U = 8;
   pdl_trigger();
+  // The router matrix is a constant of the layer: the first pass over this warp's row (the whole row for
+  // d <= 32*VEC*U) is fetched while the previous kernel in the stream is still running.
+  uint4 rw[U];
+  if (i < N) {
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if ((lane + u * 32) * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(Wr + (size_t)i * d + (lane + u * 32) * VEC);
+  }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
 #ifdef MOESPEC_ROUTE_TIMING
   const long long tm0 = clock64();
 #endif
   if (i < N) {
-    constexpr int VEC = 16 / sizeof(T);
-    constexpr int U = 8;
     const T *w = Wr + (size_t)i * d;
     float acc[TT];
 #pragma unroll
     for (int tt = 0; tt < TT; ++tt) acc[tt] = 0.f;
     for (int j0 = lane * VEC; j0 < d; j0 += 32 * VEC * U) {
-      uint4 rw[U];
+      if (j0 != lane * VEC) {
 #pragma unroll
-      for (int u = 0; u < U; ++u)
-        if (j0 + u * 32 * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(w + j0 + u * 32 * VEC);
+        for (int u = 0; u < U; ++u)
+          if (j0 + u * 32 * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(w + j0 + u * 32 * VEC);
+      }
       // two tokens per pass: their loads are all issued before the first FMA
 #pragma unroll
       for (int tt = 0; tt < TT; tt += 2) {
