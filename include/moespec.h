@@ -248,6 +248,62 @@ int moespec_last_launch_count(moespec_layer_t *layer);
 /* Free the workspace and the handle.  NULL is accepted.  Borrowed buffers are untouched. */
 int moespec_destroy(moespec_layer_t *layer);
 
+/* ---- Residual stack of budgeted MoE layers ---------------------------------
+ * The method enforces the expert budget at every MoE layer of the model
+ * (abstract; Section 4 runs 16-, 48- and 32-layer models) and names a per-layer
+ * budget as an open extension (Limitations section).  A stack chains L existing layers on
+ * one residual stream:
+ *     x_0 = hidden,   x_{l+1} = dtype( x_l + layer_l(x_l ; B_l) ),   out = x_L.
+ * Only the MoE blocks are on this path (attention and normalisation between them
+ * are not part of the method).  Every layer must have been created with
+ * residual = 1 and out_dtype equal to its dtype, on one device, with equal d and
+ * dtype; a layer may appear once.  The stack borrows the layer handles (they
+ * must outlive it, and must not run in another stream at the same time: each
+ * layer's workspace is used by its position in the pass) and owns the L-1
+ * intermediate streams, each [max_M, d] with max_M the smallest of the layers'.
+ *
+ * One pass is enqueued as ONE CUDA graph launch: the 4L kernels are captured once
+ * per (M, k, budgets, buffer pair) on an internal stream with programmatic
+ * dependent launch edges, so that each kernel's prologue (barrier set-up, tensor
+ * memory allocation, the router-matrix prefetch of the next layer) overlaps the
+ * tail of its predecessor; the cached graph is re-instantiated when an argument
+ * or a layer setting (static ranking, profiling, wait bounds) changes.  The first
+ * call with new arguments therefore allocates (graph instantiation); later calls
+ * do not.  moespec_stack_set_graph(stack, 0) enqueues the kernels one by one
+ * instead (same results). */
+typedef struct moespec_stack moespec_stack_t;
+
+/* layers: host array of n_layers (1..1024) live layer handles, first layer first.
+ * Errors: NULL_POINTER, BAD_HANDLE (a dead layer), INVALID_ARG (mismatched d,
+ * dtype, device; residual = 0; fp32 output on a 16-bit layer; repeated layer),
+ * OUT_OF_MEMORY, CUDA. */
+int moespec_stack_create(moespec_layer_t *const *layers, int n_layers, moespec_stack_t **out_stack);
+
+/* One pass.  hidden, out: device [M, d] in the layers' dtype, 16-byte aligned, not
+ * aliased.  B_per_layer: HOST array of n_layers budgets (read before returning).
+ * k as in moespec_verify_layer.  Enqueues on `stream` and returns.
+ * Errors: BAD_HANDLE (also when a member layer was destroyed), NULL_POINTER,
+ * INVALID_ARG, UNSUPPORTED (alignment), CUDA. */
+int moespec_verify_stack(moespec_stack_t *stack, const void *hidden, int M, int k, const int *B_per_layer,
+                         void *out, void *stream);
+
+/* Same pass with HOST buffers [M, d] (dtype): copy in, L layers, copy out, then
+ * synchronise.  Pinned buffers: copies and kernels are one graph launch on the
+ * internal stream, after the work already queued on `stream`. */
+int moespec_verify_stack_host(moespec_stack_t *stack, const void *hidden_host, int M, int k,
+                              const int *B_per_layer, void *out_host, void *stream);
+
+/* Copy x_l of the last pass (1 <= l <= n_layers-1; x_0 and x_L are the caller's
+ * buffers) to host_buf [M, d].  Synchronises the device.  Per-layer routing and
+ * statistics of the pass are read from the layer handles as usual. */
+int moespec_stack_get_stream(moespec_stack_t *stack, int l, void *host_buf);
+
+int moespec_stack_set_graph(moespec_stack_t *stack, int on);
+/* Kernels of the last pass (sum over its layers; one graph launch carries them all). */
+int moespec_stack_last_launch_count(moespec_stack_t *stack);
+/* Frees the intermediate streams and the graph; the layers stay alive.  NULL is accepted. */
+int moespec_stack_destroy(moespec_stack_t *stack);
+
 const char *moespec_strerror(int status);
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int moespec_last_cuda_error(void);

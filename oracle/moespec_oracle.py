@@ -312,8 +312,8 @@ def round_storage(x, dtype):
 def verify_stack(H, layers, k, budgets, policy, shortlist_mode, renormalize, storage, static_ranks=None):
     """L budgeted MoE layers on a residual stream: x_0 = H, x_{l+1} = storage(x_l + out_l(x_l)).
 
-    The budget is enforced at each MoE layer (abstract; Section 4.6 leaves a
-    per-layer budget open, so `budgets` is one B per layer).  Only the MoE blocks
+    The budget is enforced at each MoE layer (abstract); the Limitations section
+    names a per-layer budget as an extension, so `budgets` is one B per layer.  Only the MoE blocks
     are on this path: attention and normalisation between them are not part of
     the method.  `layers[l]` is a dict with router_w, router_bias, w_gate, w_up,
     w_down.  The stream is rounded to the storage dtype after every layer, as a

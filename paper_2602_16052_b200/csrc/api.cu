@@ -34,6 +34,28 @@ struct moespec_layer {
   bool graph_usable;
   long long debug_spin_limit;
   int debug_ready_bias;
+  unsigned epoch;       // bumped whenever something a captured graph has baked in changes
+};
+
+// L layers on one residual stream (the MoE blocks of a model, one after the other)
+struct moespec_stack {
+  unsigned long long magic;
+  std::vector<moespec_layer *> layers;
+  int device, d, dtype, max_M, max_k;
+  size_t row_bytes;         // d * sizeof(dtype)
+  char *arena;              // x_1 .. x_{L-1}, then the host entry point's staging buffers
+  char *in_stage, *out_stage;
+  bool graph_on, graph_usable;
+  cudaStream_t own_stream;
+  cudaEvent_t ev_in;
+  cudaGraphExec_t exec;     // one cached instantiation: (M, k, budgets, buffers, epochs)
+  int g_M, g_k;
+  std::vector<int> g_B;
+  const void *g_in;
+  void *g_out;
+  bool g_host;
+  unsigned g_epoch;
+  int last_M, last_launches;
 };
 
 namespace {
@@ -42,6 +64,8 @@ constexpr unsigned long long kMagic = 0x4d6f455370656331ULL;
 thread_local int tl_cuda_error = 0;
 std::mutex g_mu;
 std::unordered_set<moespec_layer *> g_live;
+std::unordered_set<moespec_stack *> g_live_stacks;
+constexpr unsigned long long kStackMagic = 0x4d6f455370656353ULL;
 
 int cuda_fail(cudaError_t e) {
   tl_cuda_error = (int)e;
@@ -52,6 +76,12 @@ bool is_live(moespec_layer *L) {
   if (!L) return false;
   std::lock_guard<std::mutex> lk(g_mu);
   return g_live.count(L) != 0 && L->magic == kMagic;
+}
+
+bool is_live(moespec_stack *S) {
+  if (!S) return false;
+  std::lock_guard<std::mutex> lk(g_mu);
+  return g_live_stacks.count(S) != 0 && S->magic == kStackMagic;
 }
 
 struct DeviceGuard {
@@ -275,6 +305,7 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   L->profiling = false;
   L->debug_spin_limit = 0;
   L->debug_ready_bias = 0;
+  L->epoch = 0;
   L->host_exec = nullptr;
   L->graph_usable = cudaStreamCreateWithFlags(&L->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming) == cudaSuccess;
@@ -458,6 +489,7 @@ int moespec_set_static_ranking(moespec_layer_t *L, const int *ranked_host, int n
   e = cudaMemcpy(L->ws.static_pos, pos.data(), sizeof(int) * N, cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e);
   L->ws.n_static = (int)order.size();
+  ++L->epoch;
   if (L->host_exec) {            // a captured graph has the old ordering size baked into its arguments
     cudaGraphExecDestroy(L->host_exec);
     L->host_exec = nullptr;
@@ -561,6 +593,7 @@ int moespec_debug_set_wait(moespec_layer_t *L, long long limit_cycles, int ready
   if (limit_cycles < 0 || ready_bias < 0) return MOESPEC_ERR_INVALID_ARG;
   L->debug_spin_limit = limit_cycles;
   L->debug_ready_bias = ready_bias;
+  ++L->epoch;
   if (L->host_exec) {            // a captured graph has the old values baked in
     cudaGraphExecDestroy(L->host_exec);
     L->host_exec = nullptr;
@@ -571,6 +604,7 @@ int moespec_debug_set_wait(moespec_layer_t *L, long long limit_cycles, int ready
 int moespec_set_profiling(moespec_layer_t *L, int on) {
   if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
   L->profiling = on != 0;
+  ++L->epoch;
   return MOESPEC_OK;
 }
 
@@ -637,5 +671,251 @@ const char *moespec_strerror(int status) {
 
 int moespec_last_cuda_error(void) { return tl_cuda_error; }
 int moespec_version(void) { return 100; }
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ residual stack
+namespace {
+
+void *stack_x(moespec_stack *S, int l, const void *in, void *out) {      // x_l of the current call
+  const int L = (int)S->layers.size();
+  if (l == 0) return const_cast<void *>(in);
+  if (l == L) return out;
+  return S->arena + (size_t)(l - 1) * S->max_M * S->row_bytes;
+}
+
+// every layer of the stack, in order, on `stream`: x_{l+1} = dtype(x_l + layer_l(x_l))
+int stack_enqueue(moespec_stack *S, const void *in, int M, int k, const int *B, void *out, cudaStream_t stream) {
+  const int L = (int)S->layers.size();
+  int launches = 0;
+  for (int l = 0; l < L; ++l) {
+    int rc = run_layer(S->layers[l], stack_x(S, l, in, out), M, k, B[l], stack_x(S, l + 1, in, out), stream);
+    if (rc) return rc;
+    launches += S->layers[l]->last_launches;
+  }
+  S->last_M = M;
+  S->last_launches = launches;
+  return MOESPEC_OK;
+}
+
+unsigned stack_epoch(moespec_stack *S) {
+  unsigned e = 0;
+  for (moespec_layer *L : S->layers) e = e * 31u + L->epoch;
+  return e;
+}
+
+bool stack_profiling(moespec_stack *S) {
+  for (moespec_layer *L : S->layers)
+    if (L->profiling) return true;
+  return false;
+}
+
+int stack_validate(moespec_stack *S, int M, int k, const int *B) {
+  if (!B) return MOESPEC_ERR_NULL_POINTER;
+  if (M < 0 || M > S->max_M) return MOESPEC_ERR_INVALID_ARG;
+  for (size_t l = 0; l < S->layers.size(); ++l) {
+    if (!is_live(S->layers[l])) return MOESPEC_ERR_BAD_HANDLE;       // a layer was destroyed under the stack
+    int rc = validate_call(S->layers[l], M, k, B[l]);
+    if (rc) return rc;
+  }
+  return MOESPEC_OK;
+}
+
+// Capture (or reuse) the graph of one stack pass.  host = the copies from/to pinned host buffers are
+// part of the graph.  Returns nullptr when graphs cannot be used; the caller then enqueues plainly.
+cudaGraphExec_t stack_graph(moespec_stack *S, const void *in, int M, int k, const int *B, void *out, bool host) {
+  const int L = (int)S->layers.size();
+  const unsigned epoch = stack_epoch(S);
+  bool hit = S->exec && S->g_M == M && S->g_k == k && S->g_in == in && S->g_out == out && S->g_host == host &&
+             S->g_epoch == epoch;
+  for (int l = 0; hit && l < L; ++l) hit = S->g_B[l] == B[l];
+  if (hit) return S->exec;
+  if (S->exec) {
+    cudaGraphExecDestroy(S->exec);
+    S->exec = nullptr;
+  }
+  const size_t bytes = (size_t)M * S->row_bytes;
+  const void *dev_in = host ? S->in_stage : in;
+  void *dev_out = host ? S->out_stage : out;
+  cudaGraph_t graph = nullptr;
+  cudaError_t e = cudaStreamBeginCapture(S->own_stream, cudaStreamCaptureModeThreadLocal);
+  if (e == cudaSuccess) {
+    if (host) e = cudaMemcpyAsync(S->in_stage, in, bytes, cudaMemcpyHostToDevice, S->own_stream);
+    if (e == cudaSuccess && stack_enqueue(S, dev_in, M, k, B, dev_out, S->own_stream) != MOESPEC_OK) e = cudaErrorUnknown;
+    if (e == cudaSuccess && host) e = cudaMemcpyAsync(out, S->out_stage, bytes, cudaMemcpyDeviceToHost, S->own_stream);
+    cudaError_t e2 = cudaStreamEndCapture(S->own_stream, &graph);
+    if (e == cudaSuccess) e = e2;
+  }
+  if (e == cudaSuccess) e = cudaGraphInstantiate(&S->exec, graph, 0);
+  if (graph) cudaGraphDestroy(graph);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    S->exec = nullptr;
+    S->graph_usable = false;
+    return nullptr;
+  }
+  S->g_M = M; S->g_k = k; S->g_in = in; S->g_out = out; S->g_host = host; S->g_epoch = epoch;
+  S->g_B.assign(B, B + L);
+  return S->exec;
+}
+
+}  // namespace
+
+extern "C" {
+
+int moespec_stack_create(moespec_layer_t *const *layers, int n_layers, moespec_stack_t **out_stack) {
+  if (!layers || !out_stack) return MOESPEC_ERR_NULL_POINTER;
+  if (n_layers < 1 || n_layers > 1024) return MOESPEC_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if (!is_live(layers[l])) return MOESPEC_ERR_BAD_HANDLE;
+  const moespec_layer_desc &d0 = layers[0]->desc;
+  int max_M = d0.max_M, max_k = d0.max_k;
+  for (int l = 0; l < n_layers; ++l) {
+    const moespec_layer_desc &d = layers[l]->desc;
+    if (d.device != d0.device || d.d != d0.d || d.dtype != d0.dtype) return MOESPEC_ERR_INVALID_ARG;
+    // the stream stays in the storage dtype and every layer adds its input back
+    if (!d.residual || (d.out_dtype != 0 && d.out_dtype != d.dtype)) return MOESPEC_ERR_INVALID_ARG;
+    for (int m = 0; m < l; ++m)
+      if (layers[m] == layers[l]) return MOESPEC_ERR_INVALID_ARG;     // a layer's workspace serves one position
+    if (d.max_M < max_M) max_M = d.max_M;
+    if (d.max_k < max_k) max_k = d.max_k;
+  }
+  DeviceGuard guard(d0.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  moespec_stack *S = new (std::nothrow) moespec_stack();
+  if (!S) return MOESPEC_ERR_OUT_OF_MEMORY;
+  S->magic = kStackMagic;
+  S->layers.assign(layers, layers + n_layers);
+  S->device = d0.device;
+  S->d = d0.d;
+  S->dtype = d0.dtype;
+  S->max_M = max_M;
+  S->max_k = max_k;
+  S->row_bytes = (size_t)d0.d * dtype_bytes(d0.dtype);
+  const size_t slab = (size_t)max_M * S->row_bytes;          // a multiple of 256 bytes: d % 64 == 0, 2 or 4 bytes each
+  void *p = nullptr;
+  cudaError_t e = cudaMalloc(&p, slab * (size_t)(n_layers - 1 + 2));
+  if (e != cudaSuccess) {
+    delete S;
+    cudaGetLastError();
+    return cuda_fail(e);
+  }
+  S->arena = static_cast<char *>(p);
+  S->in_stage = S->arena + slab * (size_t)(n_layers - 1);
+  S->out_stage = S->in_stage + slab;
+  S->exec = nullptr;
+  S->graph_on = true;
+  S->graph_usable = cudaStreamCreateWithFlags(&S->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
+                    cudaEventCreateWithFlags(&S->ev_in, cudaEventDisableTiming) == cudaSuccess;
+  S->last_M = 0;
+  S->last_launches = 0;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_live_stacks.insert(S);
+  }
+  *out_stack = S;
+  return MOESPEC_OK;
+}
+
+int moespec_verify_stack(moespec_stack_t *S, const void *hidden, int M, int k, const int *B_per_layer, void *out,
+                         void *stream) {
+  if (!is_live(S)) return MOESPEC_ERR_BAD_HANDLE;
+  int rc = stack_validate(S, M, k, B_per_layer);
+  if (rc) return rc;
+  if (M == 0) return MOESPEC_OK;
+  if (!hidden || !out) return MOESPEC_ERR_NULL_POINTER;
+  if (!aligned16(hidden) || !aligned16(out)) return MOESPEC_ERR_UNSUPPORTED;
+  if (hidden == out) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(S->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (S->graph_on && S->graph_usable && !stack_profiling(S)) {
+    cudaGraphExec_t g = stack_graph(S, hidden, M, k, B_per_layer, out, false);
+    if (g) {
+      cudaError_t e = cudaGraphLaunch(g, s);
+      return e == cudaSuccess ? MOESPEC_OK : cuda_fail(e);
+    }
+  }
+  return stack_enqueue(S, hidden, M, k, B_per_layer, out, s);
+}
+
+int moespec_verify_stack_host(moespec_stack_t *S, const void *hidden_host, int M, int k, const int *B_per_layer,
+                              void *out_host, void *stream) {
+  if (!is_live(S)) return MOESPEC_ERR_BAD_HANDLE;
+  int rc = stack_validate(S, M, k, B_per_layer);
+  if (rc) return rc;
+  if (M == 0) return MOESPEC_OK;
+  if (!hidden_host || !out_host) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(S->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e;
+  if (S->graph_on && S->graph_usable && !stack_profiling(S) && is_pinned(hidden_host) && is_pinned(out_host)) {
+    cudaGraphExec_t g = stack_graph(S, hidden_host, M, k, B_per_layer, out_host, true);
+    if (g) {
+      if ((e = cudaEventRecord(S->ev_in, s)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaStreamWaitEvent(S->own_stream, S->ev_in, 0)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaGraphLaunch(g, S->own_stream)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaStreamSynchronize(S->own_stream)) != cudaSuccess) return cuda_fail(e);
+      return MOESPEC_OK;
+    }
+  }
+  const size_t bytes = (size_t)M * S->row_bytes;
+  if ((e = cudaMemcpyAsync(S->in_stage, hidden_host, bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess) return cuda_fail(e);
+  rc = stack_enqueue(S, S->in_stage, M, k, B_per_layer, S->out_stage, s);
+  if (rc) return rc;
+  if ((e = cudaMemcpyAsync(out_host, S->out_stage, bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+  return MOESPEC_OK;
+}
+
+int moespec_stack_get_stream(moespec_stack_t *S, int l, void *host_buf) {
+  if (!is_live(S)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!host_buf) return MOESPEC_ERR_NULL_POINTER;
+  if (l < 1 || l >= (int)S->layers.size()) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(S->device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (S->last_M > 0) {
+    e = cudaMemcpy(host_buf, S->arena + (size_t)(l - 1) * S->max_M * S->row_bytes, (size_t)S->last_M * S->row_bytes,
+                   cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return MOESPEC_OK;
+}
+
+int moespec_stack_set_graph(moespec_stack_t *S, int on) {
+  if (!is_live(S)) return MOESPEC_ERR_BAD_HANDLE;
+  S->graph_on = on != 0;
+  return MOESPEC_OK;
+}
+
+int moespec_stack_last_launch_count(moespec_stack_t *S) {
+  if (!is_live(S)) return MOESPEC_ERR_BAD_HANDLE;
+  return S->last_launches;
+}
+
+int moespec_stack_destroy(moespec_stack_t *S) {
+  if (!S) return MOESPEC_OK;
+  {
+    std::lock_guard<std::mutex> lk(g_mu);
+    if (g_live_stacks.erase(S) == 0) return MOESPEC_ERR_BAD_HANDLE;
+  }
+  int rc = MOESPEC_OK;
+  {
+    DeviceGuard guard(S->device);
+    if (S->exec) cudaGraphExecDestroy(S->exec);
+    if (S->graph_usable) {
+      cudaEventDestroy(S->ev_in);
+      cudaStreamDestroy(S->own_stream);
+    }
+    cudaError_t e = cudaFree(S->arena);
+    if (e != cudaSuccess) rc = cuda_fail(e);
+  }
+  S->magic = 0;
+  delete S;
+  return rc;
+}
 
 }  // extern "C"

@@ -31,7 +31,9 @@ EXPORTS = [
     "moespec_layer_create", "moespec_verify_layer", "moespec_verify_layer_host",
     "moespec_calibrate", "moespec_get_static_counts", "moespec_set_static_ranking", "moespec_reset_calibration",
     "moespec_route_from_logits", "moespec_route_static", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
-    "moespec_debug_set_wait", "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy", "moespec_strerror", "moespec_last_cuda_error",
+    "moespec_debug_set_wait", "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy",
+    "moespec_stack_create", "moespec_verify_stack", "moespec_verify_stack_host", "moespec_stack_get_stream",
+    "moespec_stack_set_graph", "moespec_stack_last_launch_count", "moespec_stack_destroy", "moespec_strerror", "moespec_last_cuda_error",
     "moespec_version",
 ]
 
@@ -93,6 +95,13 @@ def lib() -> C.CDLL:
         L.moespec_get_kernel_times.argtypes = [vp, vp, ci, vp]
         L.moespec_last_launch_count.argtypes = [vp]
         L.moespec_destroy.argtypes = [vp]
+        L.moespec_stack_create.argtypes = [vp, ci, C.POINTER(vp)]
+        L.moespec_verify_stack.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+        L.moespec_verify_stack_host.argtypes = [vp, vp, ci, ci, vp, vp, vp]
+        L.moespec_stack_get_stream.argtypes = [vp, ci, vp]
+        L.moespec_stack_set_graph.argtypes = [vp, ci]
+        L.moespec_stack_last_launch_count.argtypes = [vp]
+        L.moespec_stack_destroy.argtypes = [vp]
         L.moespec_strerror.argtypes = [ci]
         L.moespec_strerror.restype = C.c_char_p
         for name in EXPORTS:
@@ -295,6 +304,74 @@ class Layer:
             code = lib().moespec_destroy(self._h)
             self._h = None
             _check(code, "moespec_destroy")
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+class Stack:
+    """L layers on one residual stream: moespec_stack_create / moespec_verify_stack / moespec_stack_destroy.
+
+    The layers are borrowed (kept referenced here); each must have residual=True and out_dtype == dtype.
+    """
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        arr = (C.c_void_p * len(self.layers))(*[L._h for L in self.layers])
+        h = C.c_void_p()
+        _check(lib().moespec_stack_create(C.cast(arr, C.c_void_p), len(self.layers), C.byref(h)), "moespec_stack_create")
+        self._h = h
+        self._last_M = 0
+
+    def _budgets(self, budgets):
+        if isinstance(budgets, int):
+            budgets = [budgets] * len(self.layers)
+        if len(budgets) != len(self.layers):
+            raise ValueError("one budget per layer")
+        return (C.c_int * len(self.layers))(*[int(b) for b in budgets])
+
+    def verify_stack(self, hidden: torch.Tensor, k: int, budgets, out: Optional[torch.Tensor] = None, stream=None):
+        M = hidden.shape[0]
+        if out is None:
+            out = torch.empty_like(hidden)
+        b = self._budgets(budgets)
+        _check(lib().moespec_verify_stack(self._h, hidden.data_ptr(), M, k, C.cast(b, C.c_void_p), out.data_ptr(),
+                                          _stream_ptr(stream)), "moespec_verify_stack")
+        self._last_M = M
+        for L in self.layers:
+            L._last = (M, k)
+        return out
+
+    def verify_stack_host(self, hidden_host: torch.Tensor, k: int, budgets, out_host: torch.Tensor, stream=None):
+        M = hidden_host.shape[0]
+        b = self._budgets(budgets)
+        _check(lib().moespec_verify_stack_host(self._h, hidden_host.data_ptr(), M, k, C.cast(b, C.c_void_p),
+                                               out_host.data_ptr(), _stream_ptr(stream)), "moespec_verify_stack_host")
+        self._last_M = M
+        for L in self.layers:
+            L._last = (M, k)
+        return out_host
+
+    def get_stream(self, l: int) -> torch.Tensor:
+        """x_l of the last pass (1 <= l <= L-1) as a CPU tensor [M, d]."""
+        x = torch.empty((self._last_M, self.layers[0].d), dtype=self.layers[0].dtype)
+        _check(lib().moespec_stack_get_stream(self._h, l, x.data_ptr()), "moespec_stack_get_stream")
+        return x
+
+    def set_graph(self, on: bool):
+        _check(lib().moespec_stack_set_graph(self._h, int(on)), "moespec_stack_set_graph")
+
+    def last_launch_count(self) -> int:
+        return lib().moespec_stack_last_launch_count(self._h)
+
+    def destroy(self):
+        if getattr(self, "_h", None) is not None and self._h:
+            code = lib().moespec_stack_destroy(self._h)
+            self._h = None
+            _check(code, "moespec_stack_destroy")
 
     def __del__(self):
         try:

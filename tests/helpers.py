@@ -26,11 +26,11 @@ def f64(t):
     return t.to("cpu", torch.float64).numpy()
 
 
-def oracle_run(case, k, B, policy, mode, renorm, logits=None):
+def oracle_run(case, k, B, policy, mode, renorm, logits=None, static_rank=None):
     return orc.verify_layer(f64(case["hidden"]), f64(case["router_w"]),
                             None if case["router_bias"] is None else f64(case["router_bias"]),
                             LazyF64(case["w_gate"]), LazyF64(case["w_up"]), LazyF64(case["w_down"]),
-                            k, B, policy, mode, renorm, logits=logits)
+                            k, B, policy, mode, renorm, logits=logits, static_rank=static_rank)
 
 
 def oracle_route(logits, k, B, policy, mode, renorm):
