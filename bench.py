@@ -190,6 +190,82 @@ def kernel_profile(layers, hiddens, outs, k, B, reps):
     return {name: sum(v) / len(v) for name, v in acc.items()}
 
 
+def time_stack(cfg, M, B, device, reps):
+    """L-layer residual stack (bf16 stream): microseconds per layer through the stack entry point (one graph
+    launch per pass), through the same entry point enqueuing kernel by kernel, and as L separate layer
+    calls; plus the share of the event-bracketed kernel time that goes to choosing experts."""
+    from paper_2602_16052_b200 import moespec
+    L = cfg.n_layers
+    weights = [synth.gen_layer(cfg, seed=2000, layer=l, device=device) for l in range(L)]
+    layers = [moespec.Layer(w["router_w"], w["router_bias"], w["w_gate"], w["w_up"], w["w_down"], max_M=M,
+                            max_k=cfg.k, policy=moespec.SUBSTITUTION, shortlist=moespec.FROM_ALL, renormalize=True,
+                            residual=True) for w in weights]
+    stack = moespec.Stack(layers)
+    x0 = synth.gen_hidden(cfg, M, seed=2000, layer=0, device=device)
+    out = torch.empty_like(x0)
+    bufs = [torch.empty_like(x0) for _ in range(2)]
+    budgets = [B] * L
+
+    def by_calls():
+        cur = x0
+        for l, lay in enumerate(layers):
+            lay.verify_layer(cur, cfg.k, B, bufs[l % 2])
+            cur = bufs[l % 2]
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3 / (reps * L)
+
+    us_graph = timed(lambda: stack.verify_stack(x0, cfg.k, budgets, out))
+    # host-side cost of enqueuing one pass (the call returns once the work is queued)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    stack.verify_stack(x0, cfg.k, budgets, out)
+    enqueue_graph_us = (time.perf_counter() - t0) * 1e6
+    torch.cuda.synchronize()
+    stack.set_graph(False)
+    us_plain = timed(lambda: stack.verify_stack(x0, cfg.k, budgets, out))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    stack.verify_stack(x0, cfg.k, budgets, out)
+    enqueue_plain_us = (time.perf_counter() - t0) * 1e6
+    torch.cuda.synchronize()
+    stack.set_graph(True)
+    us_calls = timed(by_calls)
+    act = sum(lay.get_stats()["n_active"] for lay in layers) / L
+    # per-kernel times of one pass with event bracketing (outside the timed runs)
+    acc = {}
+    for lay in layers:
+        lay.set_profiling(True)
+    for _ in range(3):
+        cur = x0
+        for l, lay in enumerate(layers):
+            lay.verify_layer(cur, cfg.k, B, bufs[l % 2])
+            cur = bufs[l % 2]
+            for name, ms_ in lay.get_kernel_times().items():
+                acc[name] = acc.get(name, 0.0) + ms_
+    tot = sum(acc.values())
+    line = {"layers": L, "M": M, "B": B, "us_per_layer_graph": us_graph, "us_per_layer_kernel_by_kernel": us_plain,
+            "us_per_layer_separate_calls": us_calls, "host_enqueue_us_per_pass_graph": enqueue_graph_us,
+            "host_enqueue_us_per_pass_kernel_by_kernel": enqueue_plain_us, "gpu_launches_per_pass": stack.last_launch_count(),
+            "n_active_mean": act, "kernel_share": {n: v / tot for n, v in acc.items()},
+            "selection_share_of_layer": (tot - acc.get("ffn", 0.0)) / tot}
+    stack.destroy()
+    for lay in layers:
+        lay.destroy()
+    del layers, weights
+    torch.cuda.empty_cache()
+    return line
+
+
 def run_tables(args, device):
     """Sweeps over every workload shape (not part of the default run): one JSON line per point."""
     from paper_2602_16052_b200 import moespec
@@ -206,16 +282,14 @@ def run_tables(args, device):
         layers = [moespec.Layer(w["router_w"], w["router_bias"], w["w_gate"], w["w_up"], w["w_down"], max_M=max_M,
                                 max_k=cfg.k, policy=moespec.SUBSTITUTION, shortlist=moespec.FROM_ALL, renormalize=True,
                                 residual=L > 1, out_dtype=out_dtype) for w in weights]
+        stack = moespec.Stack(layers) if L > 1 else None
         for M in Ms:
             x0 = synth.gen_hidden(cfg, M, seed=2000, layer=0, device=device)
             bufs = [torch.empty_like(x0, dtype=out_dtype) for _ in range(2)]
             for B in Bs:
                 def one_pass():
-                    if L > 1:        # stack: x <- dtype(x + MoE_l(x)), layer after layer
-                        cur = x0
-                        for l, lay in enumerate(layers):
-                            lay.verify_layer(cur, cfg.k, B, bufs[l % 2])
-                            cur = bufs[l % 2]
+                    if L > 1:        # stack: x <- dtype(x + MoE_l(x)), all layers as one graph launch
+                        stack.verify_stack(x0, cfg.k, [B] * L, bufs[0])
                     else:            # single layer: rotate over independently seeded copies
                         for lay in layers:
                             lay.verify_layer(x0, cfg.k, B, bufs[0])
@@ -244,6 +318,8 @@ def run_tables(args, device):
                                   "n_active": round(act, 2), "n_union": round(uni, 2), "MB": round(by / 1e6, 1),
                                   "GBs": round(by / us / 1e3, 1), "frac_of_" + peak_kind: round(by / us / 1e3 / peak, 3),
                                   "ideal_us": round(by / peak / 1e3, 1)}), flush=True)
+        if stack is not None:
+            stack.destroy()
         for lay in layers:
             lay.destroy()
         del layers, weights
@@ -482,6 +558,11 @@ def main():
         for SL in st_layers:
             SL.destroy()
 
+    # the 16-layer stack of the same shape: one graph launch per pass against layer-by-layer calls
+    stack_line = None
+    if not args.no_sweep:
+        stack_line = time_stack(synth.CONFIGS["olmoe16"], M, B, device, max(3, args.steps // 64))
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         us, cores, reps = time_oracle(cfg, M, B, 10.0, 6)
@@ -507,6 +588,7 @@ def main():
             "sweep": sweep,
             "static_ranking": static_line,
             "raw_gating": raw_line,
+            "stack": stack_line,
             "fit_time_vs_active_experts": fit,
             "read_stream_GBs_torch_sum": read_stream_gbs,
         }

@@ -148,7 +148,7 @@ CONFIGS = {
 SWEEPS = {
     "tiny":    {"M": [15], "B": [8]},
     "olmoe":   {"M": [63], "B": [16, 32, 48, 64]},
-    "olmoe16": {"M": [1, 7, 31, 63, 127, 255], "B": [32, 64]},
+    "olmoe16": {"M": [1, 7, 31, 63, 127, 255, 511], "B": [32, 64]},
     "qwen3":   {"M": [63, 127], "B": [32, 64, 128]},
     "mixtral": {"M": [15, 63], "B": [4, 6, 8]},
 }

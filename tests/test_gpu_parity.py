@@ -192,6 +192,14 @@ def test_token_chunking_beyond_256_rows_per_expert():
     assert max(r["count"]) == 300
 
 
+def test_largest_tree_of_the_sweep_511_tokens():
+    # d, N, k of the OLMoE-shaped layer at the largest tree size of the stack sweep; popular experts get
+    # several 128-row token chunks, the tail experts a handful of rows
+    cfg = synth.CONFIGS["olmoe"].with_(f=256)
+    out, r, st = run_e2e(cfg, 511, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    assert max(r["count"]) > 256 and st["n_rows"] == 511 * cfg.k
+
+
 def test_qwen3_shape_layer():
     cfg = synth.CONFIGS["qwen3"]
     for M, B in ((63, 32), (127, 128)):
