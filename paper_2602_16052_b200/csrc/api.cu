@@ -147,6 +147,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.colmask, N * (size_t)w.mask_words);
   c.take(w.arrive, M);
   c.take(w.arrive_route, 4);
+  c.take(w.early_flag, 4);
   c.take(w.calib_count, N);
   c.take(w.static_pos, N);
   w.n_static = 0;
@@ -187,7 +188,10 @@ bool is_pinned(const void *p) {
 
 int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
-  if (L->use_tc) c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
+  if (L->use_tc) {
+    c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
+    c.early = tc_early_start(L->desc, M) ? 1 : 0;
+  }
   c.debug_spin_limit = L->debug_spin_limit;
   c.debug_ready_bias = L->debug_ready_bias;
   int launches = 0;
@@ -295,6 +299,7 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
     int cu_res = 0;
     e = tc_encode_maps(d, L->ws, L->R_cap, &L->maps, &cu_res);
     if (e == cudaSuccess) e = tc_configure();
+    if (e == cudaSuccess) e = routing_configure();
     if (e != cudaSuccess) {
       cudaFree(L->arena);
       delete L;

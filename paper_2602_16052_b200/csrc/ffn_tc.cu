@@ -57,7 +57,7 @@ constexpr int kBRegionMax = 16 * 1024;           // token-row bytes per stage: 8
 constexpr int kMmaTail = 16 * 1024;              // an M=128 MMA reads 16 KB from the start of a (possibly shorter) slab
 constexpr int kMaxStages = 8;
 constexpr int kSmemBudget = 227 * 1024;
-constexpr int kCtrlBytes = 512;                  // barriers, unit queue, TMEM base, abort flag
+constexpr int kCtrlBytes = 1024;                 // barriers, unit queue, TMEM base, abort flag, token->row table
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kSpinLimitCycles = 2000000000LL;   // default bound of every wait: ~1 s at 2 GHz
 
@@ -89,6 +89,12 @@ struct TcArgs {
   void *out;            // [M, d] bf16 or fp32
   int M, k, residual, out_is_fp32;
   long long spin_limit; // cycles after which any wait gives up
+  // early start (see the kernel's header comment)
+  int early;                 // 1: CTA c begins with gate/up unit c of the shortlist before routing has finished
+  const int *early_flag;     // 0 until the routing kernel has published the shortlist, then |S| + 1
+  const int *S_rank;         // shortlist in rank order
+  const int *perm_row2tok;   // gather order: row -> token
+  int tiles_real;            // f / ru: gate/up units per expert
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -234,6 +240,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(ctrl_gen + kMiscOff);
   volatile int *abort_flag = reinterpret_cast<volatile int *>(ctrl_gen + kMiscOff + 4);
   Unit *q_unit = reinterpret_cast<Unit *>(ctrl_gen + 256);       // [kQueue] x 32 bytes
+  int *tok2row = reinterpret_cast<int *>(ctrl_gen + 512);        // [128] token -> row of h_mid (early units)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_stages = a.n_stages;
@@ -266,8 +273,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // everything above overlaps the tail of the previous kernel; its results are read from here on
-  pdl_wait();
+  // Everything above overlaps the tail of the previous kernel.  Without early start its results are read
+  // from here on; with it each role waits at the point where it first needs them.
+  if (!a.early) pdl_wait();
 
   if (warp == 0) {
     // ===================================================== dispenser + TMA producer
@@ -276,7 +284,8 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     // CTA b starts with unit b; later units come from the dispenser.  The next unit is drawn a few
     // stages before the current one ends: early enough that the atomic and the descriptor load are
     // hidden behind the stages still in flight, late enough that no CTA sits on units others could run.
-    const int n_up = a.n_units[0], n_total = n_up + a.n_units[1];
+    int n_total = 0;                 // valid once `waited`
+    bool waited = !a.early;          // has this warp waited for the routing kernels?
     uint32_t it = 0, qi = 0;
     int ok = 1;
     const uint64_t wpol = l2_evict_first_policy();
@@ -284,11 +293,46 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     sentinel.expert = -1; sentinel.tile = 0; sentinel.row0 = 0; sentinel.n_rows = 0; sentinel.chunk = 0;
     sentinel.phase = 0; sentinel.pad0 = 0; sentinel.pad1 = 0;
     Unit un = sentinel;
-    if (lane == 0 && (int)blockIdx.x < n_total) un = a.units[blockIdx.x];
-    while (true) {
-      Unit un_next = sentinel;
-      int u_next = n_total;
+    if (a.early) {
+      // The routing kernel publishes the shortlist long before the gather order exists.  CTA c starts on
+      // gate/up unit c of the rank-ordered list (expert S_rank[c / tiles], slab c % tiles) with ALL tokens
+      // as the MMA's N dimension, read straight from `hidden`; the epilogue keeps the routed tokens only.
+      // The routing kernel builds the unit list in the same order, so unit c of the list is this unit.
       if (lane == 0) {
+        const long long t0 = clock64();
+        int fl;
+        while ((fl = ld_acquire(a.early_flag)) == 0) {
+          if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
+          __nanosleep(32);
+        }
+        if (ok && (int)blockIdx.x < (fl - 1) * a.tiles_real) {
+          un.expert = __ldcg(a.S_rank + blockIdx.x / a.tiles_real);
+          un.tile = blockIdx.x % a.tiles_real;
+          un.n_rows = a.M;
+          un.pad0 = 1;                 // dense: every token, rows of `hidden`
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (ok && !__shfl_sync(0xffffffffu, un.pad0, 0)) {      // no early unit for this CTA: wait like everybody
+        pdl_wait();
+        waited = true;
+      }
+    }
+    if (waited) {
+      n_total = a.n_units[0] + a.n_units[1];
+      if (lane == 0 && (int)blockIdx.x < n_total) un = a.units[blockIdx.x];
+    }
+    while (ok) {
+      Unit un_next = sentinel;
+      int u_next = 0x7fffffff;
+      if (lane == 0) {
+        // units without rows (an expert kept in the list only because CTAs may have started on it): nothing
+        // to stream; a down unit still counts as done
+        while (un.expert >= 0 && un.n_rows == 0 && !un.pad0) {
+          if (un.phase == 1) atomicAdd(a.down_done, 1);
+          const int u2 = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
+          un = u2 < n_total ? a.units[u2] : sentinel;
+        }
         const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
         if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
         if (ok) {
@@ -313,6 +357,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int row0 = __shfl_sync(0xffffffffu, un.row0, 0);
       const int n_rows = __shfl_sync(0xffffffffu, un.n_rows, 0);
       const int phase = __shfl_sync(0xffffffffu, un.phase, 0);
+      const int dense = __shfl_sync(0xffffffffu, un.pad0, 0);
       const int n_pad = (n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const int cps = chunks_per_stage(a, phase, n_pad);
       const int k_iters = (phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
@@ -326,13 +371,18 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int box_rows = kTokBox << bsel;
       const int t_per = n_pad / box_rows;                          // token copies per K chunk
       const int n_tok_rows = n_pad;                                // rows that arrive per K chunk
-      const CUtensorMap *map_b = phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel];
+      const CUtensorMap *map_b = dense ? &maps.hidden : (phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel]);
       const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_tok_rows * 128u;
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       for (int kc = 0; kc < k_iters; ++kc, ++it) {
         const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
         const uint32_t full = bar_full + 8 * s;
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
+        if (kc == draw_at && !waited) {        // the unit list and the gathered rows are needed from here on
+          pdl_wait();
+          waited = true;
+          n_total = a.n_units[0] + a.n_units[1];
+        }
         if (lane == 0) {
           if (kc == draw_at) u_next = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
@@ -437,12 +487,55 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag, a.spin_limit)) break;
-      tc_fence_after();
       const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
       const int ru = un.phase == 0 ? a.ru : a.ru_down;
       const int col_out = un.tile * ru + row_in_tile;       // index along f (gate/up) or d (down)
+      if (un.pad0) {
+        // Early unit: the accumulator holds the slab for EVERY token.  Routing has finished by now (this
+        // unit alone streamed for longer than the routing kernels run); its list entry says which rows of
+        // h_mid the expert owns and the gather order says which token each row is.
+        pdl_wait();
+        const int et = (int)threadIdx.x - 64;
+        Unit real = a.units[blockIdx.x];
+        if (real.expert != un.expert || real.tile != un.tile || real.phase != 0 || real.n_rows > kMaxTokChunk) {
+          if (et == 0) atomicExch(a.status, (int)MOESPEC_ERR_INTERNAL);      // the two kernels disagree on the list
+          real.n_rows = 0;
+        }
+        tok2row[et] = -1;
+        epilogue_bar();
+        if (et < real.n_rows) tok2row[__ldcg(a.perm_row2tok + real.row0 + et)] = real.row0 + et;
+        epilogue_bar();
+        if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag, a.spin_limit)) break;
+        tc_fence_after();
+        const int n_tok = quarter * 32 < ru ? un.n_rows : 0;
+        for (int c0 = 0; c0 < n_tok; c0 += 16) {
+          uint32_t g[16], up[16];
+          tc_ld16(taddr + c0, g);
+          tc_ld16(taddr + n_pad + c0, up);
+          tc_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int row = tok2row[c0 + i];          // broadcast read; -1: token not routed to this expert
+            if (row < 0) continue;
+            const float gv = __uint_as_float(g[i]);
+            const float m = __fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(up[i]);
+            if (a.is_fp16) reinterpret_cast<__half *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2half_rn(m);
+            else reinterpret_cast<__nv_bfloat16 *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2bfloat16_rn(m);
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(bar_acc_empty + 8 * ab);
+        __threadfence();
+        fence_proxy_async();
+        epilogue_bar();
+        if (threadIdx.x == 64) atomicAdd(a.ready + real.chunk, 1);
+        mbar_arrive(bar_q_empty + 8 * q);
+        ++acc_it;
+        continue;
+      }
+      if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag, a.spin_limit)) break;
+      tc_fence_after();
       const int n_live = quarter * 32 < ru ? un.n_rows : 0;     // accumulator lanes beyond the slab hold nothing
       // One warp per scheduler runs this loop, so it is latency-bound: the sixteen columns of a step are
       // computed as independent chains (approximate exp and divide: two instructions each, error far
@@ -504,6 +597,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 
+  if (a.early) pdl_wait();      // threads that have not needed the routing results so far
   // ===================================================== combine
   // out_t = sum over the kept slots of wgt[t, slot] * y[row(t, slot)], slots in a fixed order; a token
   // with no kept expert gets exact zeros (Section 3.3).  Needs every down unit of the call.
@@ -585,12 +679,18 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static cudaError_t get_encode_fn(EncodeTiledFn *fn) {
+  static EncodeTiledFn cached = nullptr;      // the entry point does not change within a process
+  if (cached) {
+    *fn = cached;
+    return cudaSuccess;
+  }
   void *p = nullptr;
   cudaDriverEntryPointQueryResult q;
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q);
   if (e != cudaSuccess) return e;
   if (q != cudaDriverEntryPointSuccess || !p) return cudaErrorNotSupported;
-  *fn = reinterpret_cast<EncodeTiledFn>(p);
+  cached = reinterpret_cast<EncodeTiledFn>(p);
+  *fn = cached;
   return cudaSuccess;
 }
 
@@ -638,6 +738,12 @@ cudaError_t tc_configure() {
   return cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget);
 }
 
+// Early start needs every token in one MMA (N <= 128) and is an option of the tensor-core path.
+bool tc_early_start(const moespec_layer_desc &d, int M) {
+  static const bool off = [] { const char *v = getenv("MOESPEC_NO_EARLY"); return v && v[0] == '1'; }();
+  return !off && is_16bit(d.dtype) && M >= 1 && M <= kMaxTokChunk;
+}
+
 static int sm_count_cached(int device) {
   static int cached[64] = {0};
   if (device < 64 && cached[device]) return cached[device];
@@ -646,6 +752,8 @@ static int sm_count_cached(int device) {
   if (device < 64) cached[device] = n;
   return n;
 }
+
+int tc_grid_size(int device) { return sm_count_cached(device); }
 
 int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
   // Measured on B200: 128-row slabs stream fastest (each unit re-reads its expert's token rows, so
@@ -702,7 +810,37 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.k = c.k;
   a.residual = D.residual;
   a.out_is_fp32 = (D.out_dtype ? D.out_dtype : D.dtype) == MOESPEC_FP32;
+  a.early = c.early;
+  a.early_flag = c.ws->early_flag;
+  a.S_rank = c.ws->S_rank;
+  a.perm_row2tok = c.ws->perm_row2tok;
+  a.tiles_real = D.f / ru;
   TcMapsCall m;
+  if (a.early) {
+    // the call's input as a TMA tensor [M, d]: rows beyond M read as zeros
+    if (maps->hidden_ptr != hidden || maps->hidden_M != c.M) {
+      EncodeTiledFn enc = nullptr;
+      cudaError_t e = get_encode_fn(&enc);
+      if (e != cudaSuccess) return e;
+      const int n_pad = (c.M + kTokBox - 1) / kTokBox * kTokBox;
+      const int box_rows = n_pad == 128 ? 128 : (n_pad % 64 == 0 ? 64 : 32);
+      const cuuint64_t dims[2] = {(cuuint64_t)D.d, (cuuint64_t)c.M};
+      const cuuint64_t strides[1] = {(cuuint64_t)D.d * 2};
+      const cuuint32_t box[2] = {kChunkK, (cuuint32_t)box_rows};
+      const cuuint32_t ones[2] = {1, 1};
+      const CUresult r = enc(&maps->hidden_map, D.dtype == MOESPEC_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16
+                                                                        : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                             2, const_cast<void *>(hidden), dims, strides, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+      if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+      maps->hidden_ptr = hidden;
+      maps->hidden_M = c.M;
+    }
+    m.hidden = maps->hidden_map;
+  } else {
+    m.hidden = maps->x_perm[0];      // unused
+  }
   m.w_gate = maps->w_gate[ri];
   m.w_up = maps->w_up[ri];
   m.w_down = maps->w_down[a.ru_down == 128 ? 0 : a.ru_down == 64 ? 1 : 2];

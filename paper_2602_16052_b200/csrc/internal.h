@@ -54,6 +54,7 @@ struct Workspace {
   unsigned *colmask;    // [N, ceil(max_M/32)] bit t of row i: expert i in A(t)
   int *arrive;          // [max_M] arrival counters of router_topk_kernel's token tiles
   int *arrive_route;    // [1] arrival counter of route_kernel's CTAs
+  int *early_flag;      // [1] 0 until the shortlist of the call is published, then |S| + 1 (may be null)
   int mask_words;       // ceil(max_M / 32)
   long long *calib_count;   // [N] Eq. 4 calibration counts c_i
   int *static_pos;          // [N] position of expert i in the fixed ordering (INT_MAX: not listed)
@@ -78,6 +79,7 @@ struct LaunchCtx {
   int R_cap;            // max_M * max_k
   cudaStream_t stream;
   int ru;               // weight rows per tensor-core work unit for this call (0: CUDA-core path)
+  int early = 0;        // 1: the FFN kernel starts on the shortlist before routing has finished (see ffn_tc.cu)
   long long debug_spin_limit = 0;   // test hook: bound of device-side waits in cycles (0 = default)
   int debug_ready_bias = 0;         // test hook: extra slabs every down unit waits for (never reported)
 };
@@ -117,19 +119,27 @@ cudaError_t launch_route(const LaunchCtx &c, const float *logits);   // softmax/
 cudaError_t launch_route_after_router(const LaunchCtx &c);           // route kernel only
 cudaError_t launch_calib_accumulate(const LaunchCtx &c);             // c_i += natural counts of the last router launch
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
+cudaError_t routing_configure();   // one-time function attributes of the routing kernels (tensor-core path)
 // ffn_simple.cu
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down
 // ffn_tc.cu
 struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 32
   CUtensorMap w_gate[3], w_up[3], w_down[3];
   CUtensorMap x_perm[3], h_mid[3];   // token-row boxes of 32, 64 and 128 rows
+  // the last call's input tensor (early-start mode): re-encoded when the pointer or M changes
+  mutable CUtensorMap hidden_map;
+  mutable const void *hidden_ptr = nullptr;
+  mutable int hidden_M = 0;
 };
 struct TcMapsCall {        // per launch: the weight maps of the chosen slab heights
   CUtensorMap w_gate, w_up, w_down;
   CUtensorMap x_perm[3], h_mid[3];
+  CUtensorMap hidden;      // the call's [M, d] input as token-row boxes (early-start mode only)
 };
 int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // gate/up slab height for a call
 int tc_rows_per_down_unit(int ru);                                         // down slab height for a call
+int tc_grid_size(int device);                                              // CTAs of the FFN kernel (one per SM)
+bool tc_early_start(const moespec_layer_desc &d, int M);                  // does a call of M tokens use early start?
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes

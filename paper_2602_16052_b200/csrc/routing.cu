@@ -150,7 +150,8 @@ template <typename T, int TT>
 __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                           const float *__restrict__ bias, float *logits,
                                                           double *prob, int *topk_idx, unsigned long long *score_fx,
-                                                          int *natcnt, int *arrive, int M, int N, int d, int k) {
+                                                          int *natcnt, int *arrive, int *early_flag, int M, int N,
+                                                          int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.y * TT;
   const int i = blockIdx.x * 8 + warp;
@@ -167,6 +168,9 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       if ((lane + u * 32) * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(Wr + (size_t)i * d + (lane + u * 32) * VEC);
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  // the call's shortlist is not known yet (the routing kernel publishes it; the FFN kernel, which can
+  // only start after this kernel has finished, polls the flag)
+  if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
 #ifdef MOESPEC_ROUTE_TIMING
   const long long tm0 = clock64();
 #endif
@@ -257,14 +261,14 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   if (c.M <= 64)
     return launch_kernel(router_topk_kernel<T, 2>, dim3(ex_tiles, (c.M + 1) / 2), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
   if (c.M <= 128)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
   return launch_kernel(router_topk_kernel<T, 8>, dim3(ex_tiles, (c.M + 7) / 8), dim3(256), 0, c.stream,
                        (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                       ws.score_fx, ws.natcnt_acc, ws.arrive, c.M, D.n_experts, D.d, c.k);
+                       ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
@@ -275,11 +279,12 @@ cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
 
 // Softmax and top-k from caller-supplied logits: one warp per token.
 __global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, double *prob, int *topk_idx,
-                                                           unsigned long long *score_fx, int *natcnt, int M, int N,
-                                                           int k) {
+                                                           unsigned long long *score_fx, int *natcnt, int *early_flag,
+                                                           int M, int N, int k) {
   const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
   pdl_trigger();
   pdl_wait();
+  if (early_flag && blockIdx.x == 0 && threadIdx.x == 0) *early_flag = 0;
   if (t < M)
     token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt,
                 threadIdx.x & 31);
@@ -305,10 +310,12 @@ struct RouteArgs {
   int policy, shortlist, renormalize;
   int tiles_up, tiles_down;     // f/RU, d/RU slabs per expert (0 when the tensor-core path is not used)
   long long expert_bytes;       // 3*d*f*sizeof(dtype)
+  int early;                    // the FFN kernel starts on the shortlist before this kernel has finished
+  int ffn_ctas;                 // CTAs of the FFN kernel: CTA c starts on gate/up unit c of the list
 };
 
 constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
-constexpr int kColmaskCache = 2048; // words of the expert x token bit matrix the last CTA keeps in shared memory
+constexpr int kColmaskCache = 1024; // words of the expert x token bit matrix the last CTA keeps in shared memory
 
 // Probability of expert `idx` from the row a warp holds in registers (lane l owns experts l, l+32, ...).
 template <int W>
@@ -407,7 +414,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   __shared__ uint32_t s_Smask[kMaskWords];
   __shared__ unsigned long long s_warp_tot[kRouteWarps];
   __shared__ int s_chunk_expert[kMaxExperts * 2];     // token chunk -> expert (first 2N chunks; more fall back)
-  __shared__ int s_nactive, s_last;
+  __shared__ int s_nactive, s_last, s_nchunks;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = a.M, N = a.N, k = a.k;
@@ -415,8 +422,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   const Workspace &ws = a.ws;
   const int t = blockIdx.x * kRouteWarps + warp;
 
-  pdl_trigger();
+  // Dependents are released only after the router kernel has completed: the FFN kernel may then start
+  // while this kernel runs, and must find the shortlist flag already reset by the router kernel.
   pdl_wait();
+  pdl_trigger();
 #ifdef MOESPEC_ROUTE_TIMING
   long long tmark[10];
   int nmark = 0;
@@ -493,6 +502,12 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   }
   __syncthreads();
   ROUTE_MARK();
+  // publish the shortlist (S_rank was written by this CTA's threads before the barrier): the FFN kernel's
+  // CTAs start streaming the weights of its best-ranked experts while the rest of the routing runs
+  if (blockIdx.x == 0 && tid == 0 && ws.early_flag) {
+    __threadfence();
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag), "r"(nS + 1) : "memory");
+  }
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
@@ -550,11 +565,37 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     }
   }
   __syncthreads();
-  ROUTE_MARK();
+  if (a.early) {
+    // Early start (M <= 128, so an expert has at most one token chunk): the unit list follows the
+    // shortlist's rank order, and the experts whose gate/up units the FFN kernel's CTAs start on before
+    // this list exists (CTA c takes unit c) keep their place even if no token was routed to them.
+    const int n_head = min((a.ffn_ctas + a.tiles_up - 1) / a.tiles_up, nS);
+    bool present = false;
+    int e_r = 0;
+    if (tid < nS) {
+      e_r = s_Srank[tid];
+      present = s_count[e_r] > 0 || tid < n_head;
+    }
+    const unsigned bal = __ballot_sync(kFull, present);
+    if (lane == 0) s_warp_tot[warp] = (unsigned long long)__popc(bal);
+    __syncthreads();
+    int pos = __popc(bal & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += (int)s_warp_tot[w];
+    if (present) {
+      s_unit_base[e_r] = pos;
+      s_chunk_expert[pos] = e_r;
+    }
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < kRouteWarps; ++w) tot += (int)s_warp_tot[w];
+      s_nchunks = tot;
+    }
+    __syncthreads();
+  }
 
   // The rest is three independent jobs, each latency-bound, run side by side:
   //   warps 0-3  row of every (token, slot)       warps 4-6  work-unit list       warp 7  coverage
-  const int n_chunks = s_unit_base[N];
+  const int n_chunks = a.early ? s_nchunks : s_unit_base[N];
   double cov = 0.0;
   if (warp < 4) {
     // rows ordered by (expert ascending, token ascending): the row of (t, e) is
@@ -609,6 +650,11 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         const int tiles = phase ? a.tiles_down : a.tiles_up;
         const int v = phase ? u - n_up : u;
         const int cpos = v / tiles;           // position in chunk-prefix space: identifies the expert
+        if (a.early) {                        // one chunk per listed expert, rank order
+          const int e1 = s_chunk_expert[cpos];
+          ws.units[u] = Unit{e1, v - cpos * tiles, s_offset[e1], s_count[e1], cpos, phase, 0, 0};
+          continue;
+        }
         int e;
         if (cpos < 2 * kMaxExperts) {
           e = s_chunk_expert[cpos];
@@ -682,6 +728,8 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.tiles_up = c.ru > 0 ? D.f / c.ru : 0;
   a.tiles_down = c.ru > 0 ? D.d / tc_rows_per_down_unit(c.ru) : 0;
   a.expert_bytes = 3LL * D.d * D.f * dtype_bytes(D.dtype);
+  a.early = c.ru > 0 ? c.early : 0;
+  a.ffn_ctas = tc_grid_size(D.device);
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
   if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);
@@ -713,7 +761,8 @@ cudaError_t launch_route_after_router(const LaunchCtx &c) { return launch_route_
 // Routing from caller-supplied logits: per-token softmax/top-k first (two launches).
 cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
   cudaError_t e = launch_kernel(softmax_topk_kernel, dim3((c.M + 3) / 4), dim3(128), 0, c.stream, logits, c.ws->prob,
-                                c.ws->topk_idx, c.ws->score_fx, c.ws->natcnt_acc, c.M, c.desc->n_experts, c.k);
+                                c.ws->topk_idx, c.ws->score_fx, c.ws->natcnt_acc, c.ws->early_flag, c.M, c.desc->n_experts,
+                                c.k);
   if (e != cudaSuccess) return e;
   return launch_route_kernel(c, logits);
 }
@@ -742,6 +791,32 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
   if (rows == 0) return cudaSuccess;
   return launch_kernel(gather_rows_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,
                        (uint4 *)c.ws->x_perm, (const int *)c.ws->perm_row2tok, (const int *)c.ws->counters, row_vec);
+}
+
+// The FFN kernel needs nearly all of an SM's shared memory.  An SM whose L1/shared split was chosen for
+// one of the small kernels above must drain before it can take such a CTA, and the small kernels sit
+// resident in their dependency waits, so the FFN kernel's CTAs could not start before the gather had
+// finished.  Asking for the largest shared-memory split here keeps the SMs in the configuration the FFN
+// kernel needs, and its CTAs become resident next to the routing kernels' CTAs.
+cudaError_t routing_configure() {
+  const int pref = (int)cudaSharedmemCarveoutMaxShared;
+  cudaError_t e = cudaSuccess;
+  auto set = [&](const void *fn) {
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, pref);
+  };
+  set((const void *)router_topk_kernel<__nv_bfloat16, 2>);
+  set((const void *)router_topk_kernel<__nv_bfloat16, 4>);
+  set((const void *)router_topk_kernel<__nv_bfloat16, 8>);
+  set((const void *)router_topk_kernel<__half, 2>);
+  set((const void *)router_topk_kernel<__half, 4>);
+  set((const void *)router_topk_kernel<__half, 8>);
+  set((const void *)softmax_topk_kernel);
+  set((const void *)route_kernel<1>);
+  set((const void *)route_kernel<2>);
+  set((const void *)route_kernel<4>);
+  set((const void *)route_kernel<8>);
+  set((const void *)gather_rows_kernel);
+  return e;
 }
 
 }  // namespace moespec

@@ -428,6 +428,38 @@ def test_static_ranking_calibration_and_layer():
     layer.destroy()
 
 
+def test_shortlisted_experts_without_rows_are_started_on_and_dropped():
+    """The FFN kernel starts on the best-ranked shortlist experts before routing has finished.  Here the
+    fixed ordering puts experts first that no token routes to (truncation keeps only the members of S inside T_k), so those
+    early units find no rows: nothing of them may reach the output, and the other experts must be complete."""
+    m = ms()
+    cfg = synth.CONFIGS["olmoe"].with_(f=256, slope=3.0)     # steep tail: many experts are in no top-k
+    case = H.make_case(cfg, 63, seed=23)
+    probe = make_layer(case, 63, cfg.k, out_dtype=torch.float32)
+    probe.verify_layer(case["hidden"], cfg.k, cfg.n_experts)
+    torch.cuda.synchronize()
+    count = probe.get_routing()["count"]
+    probe.destroy()
+    unused = [e for e in range(cfg.n_experts) if count[e] == 0]
+    used = [e for e in range(cfg.n_experts) if count[e] > 0]
+    assert len(unused) >= 6, "fixture should leave experts outside every top-k"
+    order = unused[:6] + used                                 # six experts without rows lead the shortlist
+    for policy, opol in ((m.TRUNCATION, orc.TRUNCATION), (m.SUBSTITUTION, orc.SUBSTITUTION)):
+        layer = make_layer(case, 63, cfg.k, shortlist=m.STATIC, policy=policy, out_dtype=torch.float32)
+        layer.set_static_ranking(order)
+        for B in (6, 10, 30):
+            out = layer.verify_layer(case["hidden"], cfg.k, B)
+            torch.cuda.synchronize()
+            r = H.oracle_run(case, cfg.k, B, opol, orc.STATIC, True, logits=layer.get_logits(), static_rank=order)
+            H.compare_routing(layer.get_routing(), r, opol, cfg.k)
+            st = layer.get_stats()
+            assert st["status"] == 0
+            if policy == m.TRUNCATION:
+                assert st["n_active"] == min(max(0, B - 6), len(used))
+            check_out(out, r["out"], cfg.dtype)
+        layer.destroy()
+
+
 # ------------------------------------------------------------------ fp16, the paper's own precision
 @pytest.mark.parametrize("ffn", ["cuda_core", "tensor_core"])
 def test_fp16_layer(ffn):
