@@ -304,6 +304,46 @@ int moespec_stack_last_launch_count(moespec_stack_t *stack);
 /* Frees the intermediate streams and the graph; the layers stay alive.  NULL is accepted. */
 int moespec_stack_destroy(moespec_stack_t *stack);
 
+/* ---- Analysis mode: oracle ranking (Eq. 6) and reconstruction error (Section 4.5) ----
+ * Not part of the verification hot path: the paper uses the oracle as an upper
+ * bound on selection quality ("requires running all experts and is impractical
+ * for speedup").
+ *
+ * moespec_oracle_ranking runs the layer unpruned on hidden [M, d] (every token
+ * keeps its natural top-k with the architecture's mixing weights, whatever the
+ * layer's policy and shortlist mode), which leaves every term
+ * c_{t,i} = g_i(h_t) E_i(h_t) of the gold output O*_t = sum_{i in T_k(h_t)} c_{t,i}
+ * in the workspace, and then selects experts greedily: starting from the empty
+ * set, n_pick times add the expert outside S that minimises
+ *     sum_t || O*_t - sum_{j in (S + i) and in T_k(h_t)} c_{t,j} ||^2
+ * (the inner sum runs over the experts the token actually routes to: the
+ * truncation output of Eq. 7 with the original weights; ties -> lower index).
+ * The loop works on the per-token k x k Gram matrices of the c_{t,i} in fp64.
+ *   order_host      [n_pick] experts in the order picked (host, written)
+ *   objective_host  [n_pick] value of the objective after each pick (host, may be NULL)
+ *   gold_energy_host sum_t ||O*_t||^2, the objective of the empty set (host, may be NULL)
+ *   out_star        device [M, d] in out_dtype: receives O* (may be NULL)
+ * The layer's routing state afterwards is that of the unpruned pass.  Allocates
+ * its scratch on the first call of the handle; synchronises `stream`.
+ * order_host can be passed to moespec_set_static_ranking of a MOESPEC_STATIC layer
+ * over the same weights to run the layer with the oracle's shortlist.
+ * Errors: BAD_HANDLE, NULL_POINTER, INVALID_ARG, UNSUPPORTED, OUT_OF_MEMORY, CUDA,
+ * or the device status of the unpruned pass. */
+int moespec_oracle_ranking(moespec_layer_t *layer, const void *hidden, int M, int k, int n_pick,
+                           int *order_host, double *objective_host, double *gold_energy_host,
+                           void *out_star, void *stream);
+
+/* Gram matrices of the last moespec_oracle_ranking call: host [M, k, k] fp64,
+ * G[t][a][b] = c_{t,a} . c_{t,b} with a, b the token's natural top-k slots in rank order. */
+int moespec_get_gram(moespec_layer_t *layer, double *gram_host);
+
+/* ||O_S - O*||_F^2 / ||O*||_F^2 over the M tokens (Section 4.5).  out_S, out_star:
+ * device [M, d] in the layer's out_dtype.  *err_host receives the ratio (0 when both
+ * are zero, +inf when only O* is); sums_host, if not NULL, the two sums
+ * {numerator, denominator}.  Fixed summation order; synchronises `stream`. */
+int moespec_reconstruction_error(moespec_layer_t *layer, const void *out_S, const void *out_star, int M,
+                                 double *err_host, double *sums_host, void *stream);
+
 const char *moespec_strerror(int status);
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int moespec_last_cuda_error(void);

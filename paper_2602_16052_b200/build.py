@@ -9,7 +9,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmoespec.so")
-SOURCES = ["api.cu", "routing.cu", "ffn_simple.cu", "ffn_tc.cu", "combine.cu", "route_static.cu"]
+SOURCES = ["api.cu", "routing.cu", "ffn_simple.cu", "ffn_tc.cu", "combine.cu", "route_static.cu", "analysis.cu"]
 HEADERS = [os.path.join(CSRC, "internal.h"), os.path.join(HERE, "..", "include", "moespec.h")]
 
 

@@ -2,6 +2,7 @@
 #include "internal.h"
 
 #include <cstdlib>
+#include <limits>
 #include <mutex>
 #include <new>
 #include <unordered_set>
@@ -35,6 +36,11 @@ struct moespec_layer {
   long long debug_spin_limit;
   int debug_ready_bias;
   unsigned epoch;       // bumped whenever something a captured graph has baked in changes
+  // analysis mode (allocated by the first moespec_oracle_ranking / moespec_reconstruction_error call)
+  char *analysis;       // gram [max_M, max_k, max_k] f64 | row2slot [R_cap] | order [N] | objective [N] f64 | sums
+  double *an_gram, *an_objective, *an_sums, *an_partial;
+  int *an_row2slot, *an_order;
+  int an_M, an_k;       // shape of the Gram matrices held
 };
 
 // L layers on one residual stream (the MoE blocks of a model, one after the other)
@@ -186,8 +192,10 @@ bool is_pinned(const void *p) {
   return at.type == cudaMemoryTypeHost;
 }
 
-int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream) {
-  LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
+int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *out, cudaStream_t stream,
+              const moespec_layer_desc *desc = nullptr) {
+  if (!desc) desc = &L->desc;      // the analysis mode runs the same weights under other routing settings
+  LaunchCtx c{desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
   if (L->use_tc) {
     c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
     c.early = tc_early_start(L->desc, M) ? 1 : 0;
@@ -311,6 +319,8 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   L->debug_spin_limit = 0;
   L->debug_ready_bias = 0;
   L->epoch = 0;
+  L->analysis = nullptr;
+  L->an_M = L->an_k = 0;
   L->host_exec = nullptr;
   L->graph_usable = cudaStreamCreateWithFlags(&L->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming) == cudaSuccess;
@@ -650,6 +660,7 @@ int moespec_destroy(moespec_layer_t *L) {
       cudaEventDestroy(L->ev_in);
       cudaStreamDestroy(L->own_stream);
     }
+    if (L->analysis) cudaFree(L->analysis);
     cudaError_t e = cudaFree(L->arena);
     if (e != cudaSuccess) rc = cuda_fail(e);
   }
@@ -921,6 +932,123 @@ int moespec_stack_destroy(moespec_stack_t *S) {
   S->magic = 0;
   delete S;
   return rc;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ analysis mode
+namespace {
+
+int analysis_alloc(moespec_layer *L) {
+  if (L->analysis) return MOESPEC_OK;
+  const moespec_layer_desc &d = L->desc;
+  Carver c;
+  auto lay = [&](char *base) {
+    c = Carver();
+    c.base = base;
+    c.take(L->an_gram, (size_t)d.max_M * d.max_k * d.max_k);
+    c.take(L->an_objective, (size_t)d.n_experts);
+    c.take(L->an_sums, 4);
+    c.take(L->an_partial, 2 * (size_t)kSqdiffParts);
+    c.take(L->an_row2slot, (size_t)L->R_cap);
+    c.take(L->an_order, (size_t)d.n_experts);
+    return (c.off + 255) & ~(size_t)255;
+  };
+  const size_t bytes = lay(nullptr);
+  void *p = nullptr;
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return cuda_fail(e);
+  }
+  L->analysis = static_cast<char *>(p);
+  lay(L->analysis);
+  return MOESPEC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int moespec_oracle_ranking(moespec_layer_t *L, const void *hidden, int M, int k, int n_pick, int *order_host,
+                           double *objective_host, double *gold_energy_host, void *out_star, void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  const moespec_layer_desc &d = L->desc;
+  if (M < 1 || M > d.max_M || k < 1 || k > d.max_k || k > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (n_pick < 1 || n_pick > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (!hidden || !order_host) return MOESPEC_ERR_NULL_POINTER;
+  if (!aligned16(hidden) || (out_star && !aligned16(out_star))) return MOESPEC_ERR_UNSUPPORTED;
+  if (out_star == hidden) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(d.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  int rc = analysis_alloc(L);
+  if (rc) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the unpruned model: every token keeps its natural top-k (B = N), no residual; O* goes to out_star
+  moespec_layer_desc full = d;
+  full.shortlist = MOESPEC_FROM_ALL;
+  full.policy = MOESPEC_SUBSTITUTION;
+  full.residual = 0;
+  void *dump = out_star ? out_star : L->ws.out_stage;
+  rc = run_layer(L, hidden, M, k, d.n_experts, dump, s, &full);
+  if (rc) return rc;
+  LaunchCtx c{&L->desc, &L->ws, M, k, d.n_experts, L->R_cap, s, 0};
+  cudaError_t e = launch_gram(c, L->an_gram, L->an_row2slot);
+  if (e == cudaSuccess)
+    e = launch_greedy(c, L->an_gram, L->an_row2slot, n_pick, L->an_order, L->an_objective, L->an_sums);
+  if (e != cudaSuccess) return cuda_fail(e);
+  L->an_M = M;
+  L->an_k = k;
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return cuda_fail(e);
+  if ((e = cudaMemcpy(order_host, L->an_order, sizeof(int) * n_pick, cudaMemcpyDeviceToHost)) != cudaSuccess)
+    return cuda_fail(e);
+  if (objective_host &&
+      (e = cudaMemcpy(objective_host, L->an_objective, sizeof(double) * n_pick, cudaMemcpyDeviceToHost)) != cudaSuccess)
+    return cuda_fail(e);
+  if (gold_energy_host &&
+      (e = cudaMemcpy(gold_energy_host, L->an_sums, sizeof(double), cudaMemcpyDeviceToHost)) != cudaSuccess)
+    return cuda_fail(e);
+  int status = 0;
+  if ((e = cudaMemcpy(&status, L->ws.status, sizeof(int), cudaMemcpyDeviceToHost)) != cudaSuccess) return cuda_fail(e);
+  return status;      // 0, or the device-side status of the unbudgeted pass
+}
+
+int moespec_get_gram(moespec_layer_t *L, double *gram_host) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  if (!gram_host) return MOESPEC_ERR_NULL_POINTER;
+  if (!L->analysis || L->an_M == 0) return MOESPEC_ERR_INVALID_ARG;
+  DeviceGuard guard(L->desc.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess)
+    e = cudaMemcpy(gram_host, L->an_gram, sizeof(double) * (size_t)L->an_M * L->an_k * L->an_k, cudaMemcpyDeviceToHost);
+  return e == cudaSuccess ? MOESPEC_OK : cuda_fail(e);
+}
+
+int moespec_reconstruction_error(moespec_layer_t *L, const void *out_S, const void *out_star, int M,
+                                 double *err_host, double *sums_host, void *stream) {
+  if (!is_live(L)) return MOESPEC_ERR_BAD_HANDLE;
+  const moespec_layer_desc &d = L->desc;
+  if (M < 1 || M > d.max_M) return MOESPEC_ERR_INVALID_ARG;
+  if (!out_S || !out_star || !err_host) return MOESPEC_ERR_NULL_POINTER;
+  DeviceGuard guard(d.device);
+  if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+  int rc = analysis_alloc(L);
+  if (rc) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  cudaError_t e = launch_sqdiff(out_S, out_star, (size_t)M * d.d, d.out_dtype ? d.out_dtype : d.dtype, L->an_partial,
+                                L->an_sums + 2, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  double sums[2] = {0.0, 0.0};
+  if (e == cudaSuccess) e = cudaMemcpy(sums, L->an_sums + 2, sizeof(sums), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (sums_host) {
+    sums_host[0] = sums[0];
+    sums_host[1] = sums[1];
+  }
+  // one division of the two device-side sums; a zero reference gives 0 (identical) or infinity
+  *err_host = sums[1] > 0.0 ? sums[0] / sums[1] : (sums[0] == 0.0 ? 0.0 : std::numeric_limits<double>::infinity());
+  return MOESPEC_OK;
 }
 
 }  // extern "C"

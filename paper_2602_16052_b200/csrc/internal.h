@@ -147,5 +147,12 @@ cudaError_t tc_configure();   // one-time function attributes
 cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const void *hidden, void *out);
 // combine.cu
 cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out);
+// analysis.cu (oracle ranking of Eq. 6, reconstruction error of Section 4.5)
+constexpr int kSqdiffParts = 64;   // slices of the squared-difference reduction
+cudaError_t launch_gram(const LaunchCtx &c, double *gram, int *row2slot);
+cudaError_t launch_greedy(const LaunchCtx &c, const double *gram, const int *row2slot, int n_pick, int *order,
+                          double *objective, double *gold_energy);
+cudaError_t launch_sqdiff(const void *a, const void *b, size_t n, int dtype, double *partial, double *out,
+                          cudaStream_t stream);
 
 }  // namespace moespec

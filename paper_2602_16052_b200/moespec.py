@@ -33,7 +33,8 @@ EXPORTS = [
     "moespec_route_from_logits", "moespec_route_static", "moespec_get_routing", "moespec_get_logits", "moespec_get_intermediate", "moespec_get_stats",
     "moespec_debug_set_wait", "moespec_set_profiling", "moespec_get_kernel_times", "moespec_last_launch_count", "moespec_destroy",
     "moespec_stack_create", "moespec_verify_stack", "moespec_verify_stack_host", "moespec_stack_get_stream",
-    "moespec_stack_set_graph", "moespec_stack_last_launch_count", "moespec_stack_destroy", "moespec_strerror", "moespec_last_cuda_error",
+    "moespec_stack_set_graph", "moespec_stack_last_launch_count", "moespec_stack_destroy",
+    "moespec_oracle_ranking", "moespec_get_gram", "moespec_reconstruction_error", "moespec_strerror", "moespec_last_cuda_error",
     "moespec_version",
 ]
 
@@ -102,6 +103,9 @@ def lib() -> C.CDLL:
         L.moespec_stack_set_graph.argtypes = [vp, ci]
         L.moespec_stack_last_launch_count.argtypes = [vp]
         L.moespec_stack_destroy.argtypes = [vp]
+        L.moespec_oracle_ranking.argtypes = [vp, vp, ci, ci, ci, vp, vp, vp, vp, vp]
+        L.moespec_get_gram.argtypes = [vp, vp]
+        L.moespec_reconstruction_error.argtypes = [vp, vp, vp, ci, vp, vp, vp]
         L.moespec_strerror.argtypes = [ci]
         L.moespec_strerror.restype = C.c_char_p
         for name in EXPORTS:
@@ -298,6 +302,35 @@ class Layer:
 
     def last_launch_count(self) -> int:
         return lib().moespec_last_launch_count(self._h)
+
+    # -- analysis mode (Eq. 6, Section 4.5)
+    def oracle_ranking(self, hidden: torch.Tensor, k: int, n_pick: int, out_star: Optional[torch.Tensor] = None,
+                       stream=None):
+        """Greedy oracle ordering: returns (order[n_pick], objective[n_pick], gold_energy)."""
+        M = hidden.shape[0]
+        order = np.zeros(n_pick, dtype=np.int32)
+        obj = np.zeros(n_pick, dtype=np.float64)
+        gold = np.zeros(1, dtype=np.float64)
+        _check(lib().moespec_oracle_ranking(self._h, hidden.data_ptr(), M, k, n_pick, _np_ptr(order), _np_ptr(obj),
+                                            _np_ptr(gold), None if out_star is None else out_star.data_ptr(),
+                                            _stream_ptr(stream)), "moespec_oracle_ranking")
+        self._last = (M, k)
+        return order.tolist(), obj, float(gold[0])
+
+    def get_gram(self) -> np.ndarray:
+        M, k = self._last
+        g = np.zeros((M, k, k), dtype=np.float64)
+        _check(lib().moespec_get_gram(self._h, _np_ptr(g)), "moespec_get_gram")
+        return g
+
+    def reconstruction_error(self, out_S: torch.Tensor, out_star: torch.Tensor, stream=None):
+        """(||O_S - O*||^2 / ||O*||^2, numerator, denominator)."""
+        err = np.zeros(1, dtype=np.float64)
+        sums = np.zeros(2, dtype=np.float64)
+        _check(lib().moespec_reconstruction_error(self._h, out_S.data_ptr(), out_star.data_ptr(), out_S.shape[0],
+                                                  _np_ptr(err), _np_ptr(sums), _stream_ptr(stream)),
+               "moespec_reconstruction_error")
+        return float(err[0]), float(sums[0]), float(sums[1])
 
     def destroy(self):
         if getattr(self, "_h", None) is not None and self._h:
