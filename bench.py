@@ -190,6 +190,39 @@ def kernel_profile(layers, hiddens, outs, k, B, reps):
     return {name: sum(v) / len(v) for name, v in acc.items()}
 
 
+def run_analysis(cfg, layer0, hidden, M, device):
+    """Reconstruction error ||O_S - O*||^2 / ||O*||^2 (Section 4.5) of router-based, static and oracle (Eq. 6)
+    shortlists at several budgets, truncation outputs, on one layer of the benchmark workload; and the time
+    of the oracle ranking itself (an unpruned pass, the Gram matrices and the greedy loop)."""
+    from paper_2602_16052_b200 import moespec
+    rw, rb, wg, wu, wd = layer0._keep
+    mk = lambda mode: moespec.Layer(rw, rb, wg, wu, wd, max_M=128, max_k=cfg.k, policy=moespec.TRUNCATION,
+                                    shortlist=mode, renormalize=True, out_dtype=torch.float32)
+    router, static, oracle = mk(moespec.FROM_ALL), mk(moespec.STATIC), mk(moespec.STATIC)
+    O_star = torch.empty((M, cfg.d), dtype=torch.float32, device=device)
+    order, obj, gold = router.oracle_ranking(hidden, cfg.k, cfg.n_experts, O_star)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(5):
+        router.oracle_ranking(hidden, cfg.k, cfg.n_experts, O_star)
+    rank_us = (time.perf_counter() - t0) / 5 * 1e6
+    for j in range(4):
+        static.calibrate(synth.gen_hidden(cfg, 128, seed=7000 + j, device=device), cfg.k)
+    static.set_static_ranking()
+    oracle.set_static_ranking(order)
+    rows = []
+    for B in (8, 16, 24, 32, 48):
+        row = {"B": B}
+        for name, lay in (("router", router), ("static", static), ("oracle", oracle)):
+            O_S = lay.verify_layer(hidden, cfg.k, B)
+            row[name] = router.reconstruction_error(O_S, O_star)[0]
+        rows.append(row)
+    for lay in (router, static, oracle):
+        lay.destroy()
+    return {"M": M, "policy": "truncation", "reconstruction_error": rows, "oracle_ranking_us": rank_us,
+            "note": "synthetic router and experts: the curves show the mechanism, not the paper's trained-model values"}
+
+
 def time_stack(cfg, M, B, device, reps):
     """L-layer residual stack (bf16 stream): microseconds per layer through the stack entry point (one graph
     launch per pass), through the same entry point enqueuing kernel by kernel, and as L separate layer
@@ -558,6 +591,11 @@ def main():
         for SL in st_layers:
             SL.destroy()
 
+    # analysis mode on the same workload: reconstruction error of the three ranking strategies (Section 4.5)
+    analysis_line = None
+    if not args.no_sweep:
+        analysis_line = run_analysis(cfg, layers[0], hiddens[0], M, device)
+
     # the 16-layer stack of the same shape: one graph launch per pass against layer-by-layer calls
     stack_line = None
     if not args.no_sweep:
@@ -589,6 +627,7 @@ def main():
             "static_ranking": static_line,
             "raw_gating": raw_line,
             "stack": stack_line,
+            "analysis": analysis_line,
             "fit_time_vs_active_experts": fit,
             "read_stream_GBs_torch_sum": read_stream_gbs,
         }

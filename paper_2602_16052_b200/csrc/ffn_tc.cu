@@ -338,15 +338,6 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         if (ok) {
           q_unit[q] = un;
           mbar_arrive(bar_q_full + 8 * q);          // release: the queue slot is visible to the consumers
-          if (un.expert >= 0 && un.phase == 1) {
-            // the rows of h_mid this unit reads are complete once every gate/up slab of the chunk is done
-            const long long t0 = clock64();
-            while (ld_acquire(a.ready + un.chunk) < a.tiles_up) {
-              if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
-              __nanosleep(64);
-            }
-            fence_proxy_async();                    // order the acquire before the TMA reads of h_mid
-          }
         }
       }
       ++qi;
@@ -374,8 +365,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const CUtensorMap *map_b = dense ? &maps.hidden : (phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel]);
       const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_tok_rows * 128u;
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
-      for (int kc = 0; kc < k_iters; ++kc, ++it) {
-        const uint32_t s = it % n_stages, ph = (it / n_stages) & 1u;
+      const int chunk = __shfl_sync(0xffffffffu, un.chunk, 0);
+      // A stage is armed and its weight copies issued by head(); its token-row copies by rows().  A down
+      // unit reads h_mid, which is complete only when every gate/up slab of its expert has been published:
+      // its first stages' weights are therefore requested BEFORE that wait, so that a CTA that runs into
+      // the dependency keeps streaming instead of idling.
+      int armed = 0;                                // stages of this unit whose barrier has been armed
+      auto head = [&](int kc) {
+        const uint32_t s = (it + kc) % n_stages, ph = ((it + kc) / n_stages) & 1u;
         const uint32_t full = bar_full + 8 * s;
         const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
         if (kc == draw_at && !waited) {        // the unit list and the gathered rows are needed from here on
@@ -389,19 +386,46 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           else mbar_expect_tx(full, tx);
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
+        if (!ok) return;
+        ++armed;
         if (lane < w_boxes) {                       // at most 8 weight copies per stage
           const int j = phase == 0 ? (lane >> 1) : lane;
           const int col = (kc * cps + j) * kChunkK;
           const CUtensorMap *mw = phase == 0 ? ((lane & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
           tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * ru, expert, wpol);
         }
+      };
+      auto rows = [&](int kc) {
+        const uint32_t s = (it + kc) % n_stages;
+        const uint32_t full = bar_full + 8 * s;
+        const uint32_t stage = smem_base + s * (uint32_t)a.stage_bytes;
         for (int tb = lane; tb < cps * t_per; tb += 32) {
           const int j = tb / t_per, r = tb - j * t_per;
           const int col = (kc * cps + j) * kChunkK;
           tma_load_2d(stage + kARegion + j * slab_bytes + r * (box_rows * 128), map_b, full, col, row0 + r * box_rows);
         }
+      };
+      int n_pre = 0;
+      if (phase == 1) {
+        n_pre = k_iters < n_stages ? k_iters : n_stages;
+        for (int kc = 0; kc < n_pre && ok; ++kc) head(kc);
+        if (ok && lane == 0) {
+          const long long t0 = clock64();
+          while (ld_acquire(a.ready + chunk) < a.tiles_up) {
+            if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
+            __nanosleep(64);
+          }
+          fence_proxy_async();                      // order the acquire before the TMA reads of h_mid
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        // on an abort the armed stages still receive their weight copies; the drain below waits for them
+        for (int kc = 0; kc < n_pre && ok; ++kc) rows(kc);
       }
+      for (int kc = n_pre; kc < k_iters && ok; ++kc) {
+        head(kc);
+        if (ok) rows(kc);
+      }
+      it += (uint32_t)armed;                        // == k_iters unless the CTA is aborting
       if (!ok) break;
       if (lane == 0 && u_next < n_total) un_next = a.units[u_next];
       un = un_next;
@@ -514,14 +538,18 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           tc_ld16(taddr + c0, g);
           tc_ld16(taddr + n_pad + c0, up);
           tc_ld_wait();
+          float m[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {               // independent chains first, as in the gathered case
+            const float gv = __uint_as_float(g[i]);
+            m[i] = __fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(up[i]);
+          }
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const int row = tok2row[c0 + i];          // broadcast read; -1: token not routed to this expert
             if (row < 0) continue;
-            const float gv = __uint_as_float(g[i]);
-            const float m = __fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(up[i]);
-            if (a.is_fp16) reinterpret_cast<__half *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2half_rn(m);
-            else reinterpret_cast<__nv_bfloat16 *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2bfloat16_rn(m);
+            if (a.is_fp16) reinterpret_cast<__half *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2half_rn(m[i]);
+            else reinterpret_cast<__nv_bfloat16 *>(a.h_mid)[(size_t)row * a.f + col_out] = __float2bfloat16_rn(m[i]);
           }
         }
         tc_fence_before();
