@@ -156,6 +156,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.early_flag, 4);
   c.take(w.calib_count, N);
   c.take(w.static_pos, N);
+  c.take(w.static_order, N);
   w.n_static = 0;
   c.take(w.units, max_chunks * (tiles_up + tiles_down));
   c.take(w.ready, max_chunks);
@@ -198,7 +199,14 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   LaunchCtx c{desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
   if (L->use_tc) {
     c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
-    c.early = tc_early_start(L->desc, M) ? 1 : 0;
+    c.early = tc_early_start(*desc, M) ? 1 : 0;
+    // The early units follow the shortlist's rank order.  Router-based ranks follow the tokens' own
+    // probabilities, so the leading experts have rows; a fixed ordering (Eq. 4) does not look at the tree,
+    // and with few tokens most of its leading experts get none: the early units would stream unused weights.
+    if (desc->shortlist == MOESPEC_STATIC) {
+      const int nS = c.B < L->ws.n_static ? c.B : L->ws.n_static;
+      if ((long long)M * k < 4LL * nS) c.early = 0;
+    }
   }
   c.debug_spin_limit = L->debug_spin_limit;
   c.debug_ready_bias = L->debug_ready_bias;
@@ -502,6 +510,8 @@ int moespec_set_static_ranking(moespec_layer_t *L, const int *ranked_host, int n
     pos[ex] = (int)r;
   }
   e = cudaMemcpy(L->ws.static_pos, pos.data(), sizeof(int) * N, cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) return cuda_fail(e);
+  e = cudaMemcpy(L->ws.static_order, order.data(), sizeof(int) * order.size(), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) return cuda_fail(e);
   L->ws.n_static = (int)order.size();
   ++L->epoch;

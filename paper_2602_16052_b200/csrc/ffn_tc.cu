@@ -32,8 +32,9 @@
 //   warp 1  lane 0: issues tcgen05.mma (kind::f16, M=128, N=n_pad, K=16) from the
 //                   stage's swizzled shared memory into TMEM; tcgen05.commit frees
 //                   the stage and finally publishes the accumulator.
-//   warps 2-5     : epilogue.  tcgen05.ld the accumulator (one TMEM lane quarter
-//                   per warp), apply SwiGLU, store to global.
+//   warps 2-9     : epilogue.  tcgen05.ld the accumulator (a TMEM lane quarter is
+//                   shared by two warps, which take alternate groups of 16
+//                   columns), apply SwiGLU, store to global.
 // The combine of the layer lives in this kernel too: after its last unit every
 // CTA waits (bounded) until all down units are stored and then produces its share
 // of `out` from y, the mixing weights and tokslot2row, adding slots in a fixed
@@ -50,7 +51,9 @@ namespace moespec {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;                      // two warps per TMEM lane quarter, each takes every other 16 columns
+constexpr int kEpiThreads = kEpiWarps * 32;
+constexpr int kThreads = 64 + kEpiThreads;       // producer warp, MMA warp, epilogue warps
 constexpr int kChunkK = 64;                      // bf16 elements per 128-byte swizzle row
 constexpr int kARegion = 32 * 1024;              // weight bytes per stage
 constexpr int kBRegionMax = 16 * 1024;           // token-row bytes per stage: 8 KB when M <= 32, else 16 KB
@@ -95,6 +98,8 @@ struct TcArgs {
   const int *S_rank;         // shortlist in rank order
   const int *perm_row2tok;   // gather order: row -> token
   int tiles_real;            // f / ru: gate/up units per expert
+  int static_nS;             // > 0: fixed shortlist (Eq. 4) of this size, known before any kernel of the call runs
+  const int *static_order;   // the fixed ordering
 };
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -221,7 +226,7 @@ __device__ __forceinline__ int ld_acquire(const int *p) {
   return v;
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
-__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
 __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_constant__ TcMapsCall maps, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -253,11 +258,11 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(bar_acc_full + 8 * b, 1);
-      mbar_init(bar_acc_empty + 8 * b, 128);
+      mbar_init(bar_acc_empty + 8 * b, kEpiThreads);
     }
     for (int q = 0; q < kQueue; ++q) {
       mbar_init(bar_q_full + 8 * q, 1);
-      mbar_init(bar_q_empty + 8 * q, 129);      // the MMA thread and the 128 epilogue threads
+      mbar_init(bar_q_empty + 8 * q, kEpiThreads + 1);      // the MMA thread and the epilogue threads
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -299,14 +304,17 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // as the MMA's N dimension, read straight from `hidden`; the epilogue keeps the routed tokens only.
       // The routing kernel builds the unit list in the same order, so unit c of the list is this unit.
       if (lane == 0) {
-        const long long t0 = clock64();
-        int fl;
-        while ((fl = ld_acquire(a.early_flag)) == 0) {
-          if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
-          __nanosleep(32);
+        int fl = a.static_nS + 1;        // a fixed shortlist needs no publication: stream from the first cycle
+        const int *rank = a.static_nS > 0 ? a.static_order : a.S_rank;
+        if (a.static_nS == 0) {
+          const long long t0 = clock64();
+          while ((fl = ld_acquire(a.early_flag)) == 0) {
+            if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
+            __nanosleep(32);
+          }
         }
         if (ok && (int)blockIdx.x < (fl - 1) * a.tiles_real) {
-          un.expert = __ldcg(a.S_rank + blockIdx.x / a.tiles_real);
+          un.expert = __ldcg(rank + blockIdx.x / a.tiles_real);
           un.tile = blockIdx.x % a.tiles_real;
           un.n_rows = a.M;
           un.pad0 = 1;                 // dense: every token, rows of `hidden`
@@ -503,6 +511,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     // ===================================================== epilogue
     const int quarter = warp & 3;           // TMEM lanes 32*quarter .. +31 belong to this warp
     const int row_in_tile = quarter * 32 + lane;
+    const int c_first = ((warp - 2) >> 2) * 16;   // the quarter's two warps interleave 16-column groups
     uint32_t acc_it = 0, qi = 0;
     while (true) {
       const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
@@ -526,14 +535,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           if (et == 0) atomicExch(a.status, (int)MOESPEC_ERR_INTERNAL);      // the two kernels disagree on the list
           real.n_rows = 0;
         }
-        tok2row[et] = -1;
+        if (et < kMaxTokChunk) tok2row[et] = -1;
         epilogue_bar();
         if (et < real.n_rows) tok2row[__ldcg(a.perm_row2tok + real.row0 + et)] = real.row0 + et;
         epilogue_bar();
         if (!mbar_wait(bar_acc_full + 8 * ab, aph, abort_flag, a.spin_limit)) break;
         tc_fence_after();
         const int n_tok = quarter * 32 < ru ? un.n_rows : 0;
-        for (int c0 = 0; c0 < n_tok; c0 += 16) {
+        for (int c0 = c_first; c0 < n_tok; c0 += 32) {
           uint32_t g[16], up[16];
           tc_ld16(taddr + c0, g);
           tc_ld16(taddr + n_pad + c0, up);
@@ -569,7 +578,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // computed as independent chains (approximate exp and divide: two instructions each, error far
       // below the 16-bit rounding of the result) before the first store is issued.
       if (un.phase == 0) {
-        for (int c0 = 0; c0 < n_live; c0 += 16) {
+        for (int c0 = c_first; c0 < n_live; c0 += 32) {
           uint32_t g[16], up[16];
           tc_ld16(taddr + c0, g);
           tc_ld16(taddr + n_pad + c0, up);
@@ -594,7 +603,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           }
         }
       } else {
-        for (int c0 = 0; c0 < n_live; c0 += 16) {
+        for (int c0 = c_first; c0 < n_live; c0 += 32) {
           uint32_t g[16];
           tc_ld16(taddr + c0, g);
           tc_ld_wait();
@@ -843,6 +852,9 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.S_rank = c.ws->S_rank;
   a.perm_row2tok = c.ws->perm_row2tok;
   a.tiles_real = D.f / ru;
+  a.static_nS = 0;
+  a.static_order = c.ws->static_order;
+  if (a.early && D.shortlist == MOESPEC_STATIC) a.static_nS = c.B < c.ws->n_static ? c.B : c.ws->n_static;
   TcMapsCall m;
   if (a.early) {
     // the call's input as a TMA tensor [M, d]: rows beyond M read as zeros

@@ -59,6 +59,7 @@ struct Workspace {
   long long *calib_count;   // [N] Eq. 4 calibration counts c_i
   int *static_pos;          // [N] position of expert i in the fixed ordering (INT_MAX: not listed)
   int n_static;             // experts in the fixed ordering (0: none set)
+  int *static_order;        // [N] the fixed ordering itself: expert at position r (first n_static entries)
   Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
   int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
   int *unit_counter;    // [0] next unit to hand out, [1] finished down units; zeroed by the route kernel

@@ -158,7 +158,6 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   __shared__ int s_last;
   constexpr int VEC = 16 / sizeof(T);
   constexpr int U = 8;
-  pdl_trigger();
   // The router matrix is a constant of the layer: the first pass over this warp's row (the whole row for
   // d <= 32*VEC*U) is fetched while the previous kernel in the stream is still running.
   uint4 rw[U];
@@ -168,6 +167,9 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       if ((lane + u * 32) * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(Wr + (size_t)i * d + (lane + u * 32) * VEC);
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  // Dependents are released only now: with a fixed shortlist the FFN kernel of this call starts at once,
+  // and it reads `hidden`, which the previous kernel in the stream may have produced.
+  pdl_trigger();
   // the call's shortlist is not known yet (the routing kernel publishes it; the FFN kernel, which can
   // only start after this kernel has finished, polls the flag)
   if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
@@ -258,11 +260,18 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   const moespec_layer_desc &D = *c.desc;
   const Workspace &ws = *c.ws;
   const int ex_tiles = (D.n_experts + 7) / 8;
-  if (c.M <= 64)
+  // With a fixed shortlist the FFN kernel streams while this kernel runs, but its CTAs only fit beside ONE
+  // router CTA per SM (registers): more tokens per CTA keep the grid within the SM count.
+  int min_tt = 2;
+  if (c.early && D.shortlist == MOESPEC_STATIC) {
+    const int sms = tc_grid_size(D.device);
+    while (min_tt < 8 && ex_tiles * ((c.M + min_tt - 1) / min_tt) > sms) min_tt *= 2;
+  }
+  if (c.M <= 64 && min_tt <= 2)
     return launch_kernel(router_topk_kernel<T, 2>, dim3(ex_tiles, (c.M + 1) / 2), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
                          ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
-  if (c.M <= 128)
+  if (c.M <= 128 && min_tt <= 4)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
                          ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
@@ -422,10 +431,17 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   const Workspace &ws = a.ws;
   const int t = blockIdx.x * kRouteWarps + warp;
 
-  // Dependents are released only after the router kernel has completed: the FFN kernel may then start
-  // while this kernel runs, and must find the shortlist flag already reset by the router kernel.
-  pdl_wait();
-  pdl_trigger();
+  // With a router-based shortlist dependents are released only after the router kernel has completed:
+  // the FFN kernel may then start while this kernel runs, and must find the shortlist flag already reset
+  // by the router kernel.  With a fixed shortlist (Eq. 4) the FFN kernel needs nothing from the router to
+  // begin streaming, so it is released at once.
+  if (a.early && a.shortlist == MOESPEC_STATIC) {
+    pdl_trigger();
+    pdl_wait();
+  } else {
+    pdl_wait();
+    pdl_trigger();
+  }
 #ifdef MOESPEC_ROUTE_TIMING
   long long tmark[10];
   int nmark = 0;
