@@ -44,7 +44,7 @@ N_COPIES = 4
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the expert-FFN launch of one
 # verify layer (M=63, B=32), from the ncu capture summarised under profiles/
-FFN_DRAM_TRAFFIC_BYTES = 409.6e6   # 404.8 MB read + 4.8 MB written (profiles/ffn_tc_kernel_olmoe_M63_B32.md)
+FFN_DRAM_TRAFFIC_BYTES = 410.0e6   # 404.8 MB read + 4.8 MB written (profiles/ffn_tc_kernel_olmoe_M63_B32.md)
 
 
 def workload_name(cfg):

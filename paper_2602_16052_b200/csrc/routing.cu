@@ -520,10 +520,8 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   ROUTE_MARK();
   // publish the shortlist (S_rank was written by this CTA's threads before the barrier): the FFN kernel's
   // CTAs start streaming the weights of its best-ranked experts while the rest of the routing runs
-  if (blockIdx.x == 0 && tid == 0 && ws.early_flag) {
-    __threadfence();
+  if (blockIdx.x == 0 && tid == 0 && ws.early_flag)      // the barrier above orders the other threads' S_rank stores before this release
     asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag), "r"(nS + 1) : "memory");
-  }
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
