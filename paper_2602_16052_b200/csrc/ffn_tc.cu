@@ -220,6 +220,13 @@ __device__ __forceinline__ int chunks_per_stage(const TcArgs &a, int phase, int 
   return p;
 }
 
+// Token rows of a unit on the MMA's N axis: 16 for the many experts that get a handful of rows (the token
+// operand is re-read by every slab of the expert and competes with the weight stream for the SM's ingest
+// rate), else a multiple of 32.
+__device__ __forceinline__ int pad_rows(int n_rows) {
+  return n_rows <= kTokBoxSmall ? kTokBoxSmall : (n_rows + kTokBox - 1) / kTokBox * kTokBox;
+}
+
 __device__ __forceinline__ int ld_acquire(const int *p) {
   int v;
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -357,7 +364,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int n_rows = __shfl_sync(0xffffffffu, un.n_rows, 0);
       const int phase = __shfl_sync(0xffffffffu, un.phase, 0);
       const int dense = __shfl_sync(0xffffffffu, un.pad0, 0);
-      const int n_pad = (n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const int n_pad = pad_rows(n_rows);
       const int cps = chunks_per_stage(a, phase, n_pad);
       const int k_iters = (phase == 0 ? a.kchunks_up : a.kchunks_down) / cps;
       const uint32_t slab_bytes = (uint32_t)n_pad * 128u;           // one K chunk of the unit's token rows
@@ -367,10 +374,13 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // Token rows arrive in as few copies as possible (the copy engine handles ~13 M boxes/s per SM,
       // so 8+ boxes per stage would cap the stream): one 128- or 64-row box when n_pad allows, else 32s.
       const int bsel = n_pad == 128 ? 2 : (n_pad % 64 == 0 ? 1 : 0);
-      const int box_rows = kTokBox << bsel;
+      const bool small = n_pad == kTokBoxSmall;
+      const int box_rows = small ? kTokBoxSmall : kTokBox << bsel;
       const int t_per = n_pad / box_rows;                          // token copies per K chunk
       const int n_tok_rows = n_pad;                                // rows that arrive per K chunk
-      const CUtensorMap *map_b = dense ? &maps.hidden : (phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel]);
+      const CUtensorMap *map_b = dense ? &maps.hidden
+                                 : small ? (phase == 0 ? &maps.x_perm16 : &maps.h_mid16)
+                                         : (phase == 0 ? &maps.x_perm[bsel] : &maps.h_mid[bsel]);
       const uint32_t tx = (uint32_t)w_boxes * sub_bytes + (uint32_t)cps * (uint32_t)n_tok_rows * 128u;
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       const int chunk = __shfl_sync(0xffffffffu, un.chunk, 0);
@@ -457,7 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const Unit un = q_unit[q];
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
-      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const int n_pad = pad_rows(un.n_rows);
       const uint32_t idesc = instr_desc_16bit(n_pad, a.is_fp16);
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
       if (!mbar_wait(bar_acc_empty + 8 * ab, aph ^ 1u, abort_flag, a.spin_limit)) break;
@@ -520,7 +530,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       ++qi;
       if (un.expert < 0) { mbar_arrive(bar_q_empty + 8 * q); break; }
       const uint32_t ab = acc_it & 1u, aph = (acc_it >> 1) & 1u;
-      const int n_pad = (un.n_rows + kTokBox - 1) / kTokBox * kTokBox;
+      const int n_pad = pad_rows(un.n_rows);
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ab * 256u;
       const int ru = un.phase == 0 ? a.ru : a.ru_down;
       const int col_out = un.tile * ru + row_in_tile;       // index along f (gate/up) or d (down)
@@ -780,6 +790,8 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
     if ((r = rows2d(&maps->x_perm[i], ws.x_perm, d.d, kTokBox << i)) != CUDA_SUCCESS) break;
     r = rows2d(&maps->h_mid[i], ws.h_mid, d.f, kTokBox << i);
   }
+  if (r == CUDA_SUCCESS) r = rows2d(&maps->x_perm16, ws.x_perm, d.d, kTokBoxSmall);
+  if (r == CUDA_SUCCESS) r = rows2d(&maps->h_mid16, ws.h_mid, d.f, kTokBoxSmall);
   if (r != CUDA_SUCCESS) {
     *cu_result = (int)r;
     return cudaErrorInvalidValue;
@@ -878,8 +890,8 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
       EncodeTiledFn enc = nullptr;
       cudaError_t e = get_encode_fn(&enc);
       if (e != cudaSuccess) return e;
-      const int n_pad = (c.M + kTokBox - 1) / kTokBox * kTokBox;
-      const int box_rows = n_pad == 128 ? 128 : (n_pad % 64 == 0 ? 64 : 32);
+      const int n_pad = c.M <= kTokBoxSmall ? kTokBoxSmall : (c.M + kTokBox - 1) / kTokBox * kTokBox;
+      const int box_rows = n_pad == 128 ? 128 : (n_pad % 64 == 0 ? 64 : (n_pad == kTokBoxSmall ? kTokBoxSmall : 32));
       const cuuint64_t dims[2] = {(cuuint64_t)D.d, (cuuint64_t)c.M};
       const cuuint64_t strides[1] = {(cuuint64_t)D.d * 2};
       const cuuint32_t box[2] = {kChunkK, (cuuint32_t)box_rows};
@@ -904,6 +916,8 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
     m.x_perm[i] = maps->x_perm[i];
     m.h_mid[i] = maps->h_mid[i];
   }
+  m.x_perm16 = maps->x_perm16;
+  m.h_mid16 = maps->h_mid16;
   const int grid = sm_count_cached(D.device);
   const size_t smem = (size_t)a.n_stages * a.stage_bytes + kMmaTail + 1024 + kCtrlBytes;
   return launch_kernel(ffn_tc_kernel, dim3(grid), dim3(kThreads), smem, c.stream, m, a);

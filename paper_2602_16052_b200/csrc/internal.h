@@ -17,6 +17,7 @@ constexpr int kMaskWords = kMaxExperts / 32;
 constexpr int kMaxK = 32;
 constexpr int kTile = 128;                 // weight rows per tensor-core work unit (MMA M)
 constexpr int kTokBox = 32;                // token rows per TMA box of the B operand
+constexpr int kTokBoxSmall = 16;           // ... for units of at most 16 rows (the smallest MMA N)
 constexpr int kMaxTokChunk = 128;          // tokens per work unit: gate and up accumulators of two units fit TMEM
 
 // One tensor-core work unit: a slab of RU (128, 64 or 32) rows of one expert's weight
@@ -127,6 +128,7 @@ cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up,
 struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 32
   CUtensorMap w_gate[3], w_up[3], w_down[3];
   CUtensorMap x_perm[3], h_mid[3];   // token-row boxes of 32, 64 and 128 rows
+  CUtensorMap x_perm16, h_mid16;     // ... and of 16 rows
   // the last call's input tensor (early-start mode): re-encoded when the pointer or M changes
   mutable CUtensorMap hidden_map;
   mutable const void *hidden_ptr = nullptr;
@@ -135,6 +137,7 @@ struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 
 struct TcMapsCall {        // per launch: the weight maps of the chosen slab heights
   CUtensorMap w_gate, w_up, w_down;
   CUtensorMap x_perm[3], h_mid[3];
+  CUtensorMap x_perm16, h_mid16;     // 16-row boxes
   CUtensorMap hidden;      // the call's [M, d] input as token-row boxes (early-start mode only)
 };
 int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // gate/up slab height for a call
