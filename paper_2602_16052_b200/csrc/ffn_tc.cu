@@ -648,15 +648,25 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   // ===================================================== combine
   // out_t = sum over the kept slots of wgt[t, slot] * y[row(t, slot)], slots in a fixed order; a token
   // with no kept expert gets exact zeros (Section 3.3).  Needs every down unit of the call.
-  // the slot table of this CTA's first work item is fetched while the last down units are still being stored
+  // Work item = one quarter of one token's columns, so that small trees still spread over the SMs; a CTA
+  // runs two items side by side when an item needs at most 128 threads (d <= 2048).  The slot tables of the
+  // first round are fetched while the last down units are still being stored.
   const int k = a.k, d = a.d;
-  int *slot_row = tok2row;                                   // [k] rows of y, then [k] mixing weights (as bits)
-  float *slot_w = reinterpret_cast<float *>(tok2row + kMaxK);
-  if ((int)blockIdx.x < a.M * 4 && (int)threadIdx.x < k) {
-    const int t = blockIdx.x >> 2;
-    slot_row[threadIdx.x] = a.tokslot2row[(size_t)t * k + threadIdx.x];
-    slot_w[threadIdx.x] = a.gate_w[(size_t)t * k + threadIdx.x];
-  }
+  const int qcols = d / 4, lanes = qcols / 4;                // float4 columns of one item
+  const int G = lanes <= 128 ? 2 : 1;                        // items per round
+  const int GT = G == 2 ? 128 : kThreads;                    // threads per item
+  const int g = (int)threadIdx.x / GT, local = (int)threadIdx.x % GT;
+  int *slot_row = tok2row;                                   // [G][kMaxK] rows of y
+  float *slot_w = reinterpret_cast<float *>(tok2row + 2 * kMaxK);   // [G][kMaxK] mixing weights
+  auto fill_tables = [&](int round) {
+    const int fg = (int)threadIdx.x / kMaxK, fs = (int)threadIdx.x % kMaxK;
+    const int item = (int)blockIdx.x + (round * G + fg) * (int)gridDim.x;
+    if (fg < G && fs < k && item < a.M * 4) {
+      slot_row[fg * kMaxK + fs] = a.tokslot2row[(size_t)(item >> 2) * k + fs];
+      slot_w[fg * kMaxK + fs] = a.gate_w[(size_t)(item >> 2) * k + fs];
+    }
+  };
+  fill_tables(0);
   if (threadIdx.x == 0 && !*abort_flag) {
     const int n_down = a.n_units[1];
     const long long t0 = clock64();
@@ -670,27 +680,26 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     if (threadIdx.x == 0) atomicExch(a.status, (int)MOESPEC_ERR_TIMEOUT);
     return;
   }
-  // work item = one quarter of one token's columns, so that small trees still spread over the SMs
-  const int qcols = d / 4;
-  for (int item = blockIdx.x; item < a.M * 4; item += gridDim.x) {
-    const int t = item >> 2, c_lo = (item & 3) * qcols;
-    if (item != (int)blockIdx.x) {                           // later items: refill the slot table
+  for (int round = 0; (int)blockIdx.x + round * G * (int)gridDim.x < a.M * 4; ++round) {
+    if (round > 0) {                                         // later rounds: refill the slot tables
       __syncthreads();
-      if ((int)threadIdx.x < k) {
-        slot_row[threadIdx.x] = a.tokslot2row[(size_t)t * k + threadIdx.x];
-        slot_w[threadIdx.x] = a.gate_w[(size_t)t * k + threadIdx.x];
-      }
+      fill_tables(round);
       __syncthreads();
     }
-    for (int c = c_lo + threadIdx.x * 4; c < c_lo + qcols; c += kThreads * 4) {
+    const int item = (int)blockIdx.x + (round * G + g) * (int)gridDim.x;
+    if (g >= G || item >= a.M * 4) continue;
+    const int t = item >> 2, c_lo = (item & 3) * qcols;
+    const int *my_row = slot_row + g * kMaxK;
+    const float *my_w = slot_w + g * kMaxK;
+    for (int c = c_lo + local * 4; c < c_lo + qcols; c += GT * 4) {
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int s0 = 0; s0 < k; s0 += 8) {
         float4 v[8];
         float w[8];
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
-          const int row = s0 + s < k ? slot_row[s0 + s] : -1;
-          w[s] = row >= 0 ? slot_w[s0 + s] : 0.f;
+          const int row = s0 + s < k ? my_row[s0 + s] : -1;
+          w[s] = row >= 0 ? my_w[s0 + s] : 0.f;
           v[s] = row >= 0 ? __ldcg(reinterpret_cast<const float4 *>(a.y + (size_t)row * d + c))
                           : make_float4(0.f, 0.f, 0.f, 0.f);
         }
