@@ -648,25 +648,22 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   // ===================================================== combine
   // out_t = sum over the kept slots of wgt[t, slot] * y[row(t, slot)], slots in a fixed order; a token
   // with no kept expert gets exact zeros (Section 3.3).  Needs every down unit of the call.
-  // Work item = one quarter of one token's columns, so that small trees still spread over the SMs; a CTA
-  // runs two items side by side when an item needs at most 128 threads (d <= 2048).  The slot tables of the
-  // first round are fetched while the last down units are still being stored.
+  // Work item = 128 consecutive columns of one token, handled by one warp (a float4 per lane): the warps of
+  // all CTAs walk the item list independently, so there is no CTA-wide barrier between items.  Lane s holds
+  // row and weight of slot s (k <= 32) and the warp shuffles them around; the first item's slots are
+  // fetched while the last down units are still being stored.
   const int k = a.k, d = a.d;
-  const int qcols = d / 4, lanes = qcols / 4;                // float4 columns of one item
-  const int G = lanes <= 128 ? 2 : 1;                        // items per round
-  const int GT = G == 2 ? 128 : kThreads;                    // threads per item
-  const int g = (int)threadIdx.x / GT, local = (int)threadIdx.x % GT;
-  int *slot_row = tok2row;                                   // [G][kMaxK] rows of y
-  float *slot_w = reinterpret_cast<float *>(tok2row + 2 * kMaxK);   // [G][kMaxK] mixing weights
-  auto fill_tables = [&](int round) {
-    const int fg = (int)threadIdx.x / kMaxK, fs = (int)threadIdx.x % kMaxK;
-    const int item = (int)blockIdx.x + (round * G + fg) * (int)gridDim.x;
-    if (fg < G && fs < k && item < a.M * 4) {
-      slot_row[fg * kMaxK + fs] = a.tokslot2row[(size_t)(item >> 2) * k + fs];
-      slot_w[fg * kMaxK + fs] = a.gate_w[(size_t)(item >> 2) * k + fs];
-    }
-  };
-  fill_tables(0);
+  const int slices = d / 128;                                // items per token
+  const int n_items = a.M * slices;
+  const int warp_global = (int)blockIdx.x + warp * (int)gridDim.x;      // consecutive items go to different SMs
+  const int warps_total = (kThreads / 32) * (int)gridDim.x;
+  int my_row = -1;
+  float my_w = 0.f;
+  if (warp_global < n_items && lane < k) {
+    const int t = warp_global / slices;
+    my_row = a.tokslot2row[(size_t)t * k + lane];
+    my_w = a.gate_w[(size_t)t * k + lane];
+  }
   if (threadIdx.x == 0 && !*abort_flag) {
     const int n_down = a.n_units[1];
     const long long t0 = clock64();
@@ -680,28 +677,25 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     if (threadIdx.x == 0) atomicExch(a.status, (int)MOESPEC_ERR_TIMEOUT);
     return;
   }
-  for (int round = 0; (int)blockIdx.x + round * G * (int)gridDim.x < a.M * 4; ++round) {
-    if (round > 0) {                                         // later rounds: refill the slot tables
-      __syncthreads();
-      fill_tables(round);
-      __syncthreads();
+  for (int item = warp_global; item < n_items; item += warps_total) {
+    const int t = item / slices, c = (item - t * slices) * 128 + lane * 4;
+    if (item != warp_global) {                               // later items: this token's slots
+      my_row = lane < k ? a.tokslot2row[(size_t)t * k + lane] : -1;
+      my_w = lane < k ? a.gate_w[(size_t)t * k + lane] : 0.f;
     }
-    const int item = (int)blockIdx.x + (round * G + g) * (int)gridDim.x;
-    if (g >= G || item >= a.M * 4) continue;
-    const int t = item >> 2, c_lo = (item & 3) * qcols;
-    const int *my_row = slot_row + g * kMaxK;
-    const float *my_w = slot_w + g * kMaxK;
-    for (int c = c_lo + local * 4; c < c_lo + qcols; c += GT * 4) {
+    {
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
       for (int s0 = 0; s0 < k; s0 += 8) {
         float4 v[8];
         float w[8];
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
-          const int row = s0 + s < k ? my_row[s0 + s] : -1;
-          w[s] = row >= 0 ? my_w[s0 + s] : 0.f;
-          v[s] = row >= 0 ? __ldcg(reinterpret_cast<const float4 *>(a.y + (size_t)row * d + c))
-                          : make_float4(0.f, 0.f, 0.f, 0.f);
+          const int row = __shfl_sync(0xffffffffu, my_row, (s0 + s) & 31);
+          const float ws = __shfl_sync(0xffffffffu, my_w, (s0 + s) & 31);
+          const bool live = s0 + s < k && row >= 0;
+          w[s] = live ? ws : 0.f;
+          v[s] = live ? __ldcg(reinterpret_cast<const float4 *>(a.y + (size_t)row * d + c))
+                      : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
         for (int s = 0; s < 8; ++s) {
