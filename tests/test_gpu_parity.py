@@ -200,6 +200,22 @@ def test_largest_tree_of_the_sweep_511_tokens():
     assert max(r["count"]) > 256 and st["n_rows"] == 511 * cfg.k
 
 
+def test_maximum_expert_count_and_k():
+    # the limits of the interface: N = 256 experts, k = 32 slots per token (every warp-wide ranking at its
+    # widest), on the tensor-core path
+    cfg = synth.LayerConfig("limits", d=256, n_experts=256, k=32, f=128, dtype="bf16", slope=1.0)
+    for B, policy in ((256, orc.SUBSTITUTION), (64, orc.SUBSTITUTION), (48, orc.TRUNCATION), (8, orc.SUBSTITUTION)):
+        run_e2e(cfg, 40, B, policy, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+
+
+def test_many_token_chunks_per_expert():
+    # 2500 tokens over 8 experts: ~5 chunks of 128 rows per expert, 40 chunks > 2N, so the unit list takes
+    # the chunk-base search path; each weight slab is re-used by all chunks of its expert
+    cfg = synth.LayerConfig("chunks", d=128, n_experts=8, k=2, f=128, dtype="bf16", slope=0.5)
+    out, r, st = run_e2e(cfg, 2500, 4, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    assert max(r["count"]) > 4 * 128 and st["n_rows"] == 2500 * 2
+
+
 def test_qwen3_shape_layer():
     cfg = synth.CONFIGS["qwen3"]
     for M, B in ((63, 32), (127, 128)):
