@@ -216,6 +216,34 @@ def test_many_token_chunks_per_expert():
     assert max(r["count"]) > 4 * 128 and st["n_rows"] == 2500 * 2
 
 
+def test_seeded_sweep_of_random_shapes_and_settings():
+    """Forty seeded draws of (N, k, M, B, d, f, dtype, policy, shortlist mode, renormalisation, residual, slope)
+    through the whole layer: the structured cases above pick their shapes by hand, this one does not."""
+    import random
+    rng = random.Random(20260216)
+    for trial in range(40):
+        N = rng.choice([2, 3, 8, 13, 32, 64, 100, 128, 200])
+        k = rng.randint(1, min(N, 12))
+        M = rng.choice([1, 2, 5, 16, 17, 33, 64, 65, 128, 129, 200])
+        B = rng.randint(1, N + 2)
+        d = rng.choice([128, 256, 384])
+        f = rng.choice([128, 256])
+        dtype = rng.choice(["bf16", "bf16", "fp16", "fp32"])
+        policy = rng.choice([orc.SUBSTITUTION, orc.TRUNCATION])
+        mode = rng.choice([orc.FROM_ALL, orc.FROM_UNION])
+        renorm = rng.random() < 0.5
+        residual = rng.random() < 0.3
+        cfg = synth.LayerConfig(f"sweep{trial}", d=d, n_experts=N, k=k, f=f, dtype=dtype,
+                                slope=rng.choice([0.0, 0.5, 1.0, 2.0]))
+        ffn = ms().FFN_CUDA_CORE if dtype == "fp32" else rng.choice([ms().FFN_TENSOR_CORE, ms().FFN_AUTO])
+        try:
+            run_e2e(cfg, M, B, policy, mode, renorm, ffn, seed=100 + trial, residual=residual,
+                    out_dtype=torch.float32)
+        except AssertionError as e:
+            raise AssertionError(f"trial {trial}: N={N} k={k} M={M} B={B} d={d} f={f} {dtype} policy={policy} "
+                                 f"mode={mode} renorm={renorm} residual={residual}: {e}") from e
+
+
 def test_qwen3_shape_layer():
     cfg = synth.CONFIGS["qwen3"]
     for M, B in ((63, 32), (127, 128)):
