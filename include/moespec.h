@@ -114,12 +114,16 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
 int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int k, int B,
                          void *out, void *stream);
 
-/* Same computation with HOST buffers: copies hidden (host [M, d]) to the device,
- * runs the layer, copies the result into out (host [M, d], out_dtype) and synchronises the
- * before returning.  With pinned (page-locked) buffers the copies and kernels are
- * captured once per (M, k, B, buffer pair) into a CUDA graph on an internal stream
- * and replayed with one launch; work already queued on `stream` is waited for
- * first.  Pageable buffers take a plain copy-launch-copy path on `stream`. */
+/* Same computation with HOST buffers: brings hidden (host [M, d]) to the device,
+ * runs the layer, delivers the result in out (host [M, d], out_dtype) and synchronises
+ * before returning.  With pinned (page-locked) buffers the whole step is captured
+ * once per (M, k, B, buffer pair) into a CUDA graph and replayed with one launch on
+ * an internal stream, after the work already queued on `stream`.  When the pinned buffers
+ * are mapped into the device's address space (the default under unified addressing)
+ * the graph has no copy nodes: a kernel pulls hidden over the interconnect into a
+ * staging buffer and the layer's last kernel writes out directly to the host buffer.
+ * Pageable buffers take a plain copy-launch-copy path on `stream`.  out_host is
+ * written only by this call and is complete when it returns. */
 int moespec_verify_layer_host(moespec_layer_t *layer, const void *hidden_host, int M, int k, int B,
                               void *out_host, void *stream);
 
