@@ -17,6 +17,7 @@
 // depend on the order in which tokens arrive and identical experts tie exactly.
 // A stand-alone softmax/top-k kernel serves callers that inject logits.
 #include "internal.h"
+#include <cstdlib>
 #include <math_constants.h>
 #include <stdio.h>
 
@@ -255,8 +256,134 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
 #endif
 }
 
+// ---------------------------------------------------------------------------
+// K1 for larger trees: the same logits, softmax and top-k, with the dot products on the tensor cores.
+// A CTA takes 16 experts x 8 tokens; its eight warps split K, each running m16n8k16 MMAs (experts on the
+// M axis, tokens on the N axis) on operands loaded straight from global memory: thread (g, tg) of a warp
+// reads 16 contiguous bytes of router rows g and g+8 and of token row g at K offset 32*step + 8*tg and
+// feeds them to two MMAs.  That assigns memory positions to the instruction's k slots in a permuted
+// order, which is immaterial for a dot product as long as both operands use the same one.  The warps'
+// partial tiles meet in shared memory and are added in warp order (a fixed order: logits are
+// reproducible), then the kernel ends like router_topk_kernel: arrival counter per token tile, softmax
+// and top-k by the CTA that completes the tile.  The CUDA-core kernel above spends its time converting and
+// multiplying element by element, which is what limits it beyond ~64 tokens.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1, __nv_bfloat16) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1, __half) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int kRmExperts = 16, kRmTokens = 8, kRmSteps = 8;     // tile of a CTA; 32-element K steps per batch
+
+template <typename T>
+__global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
+                                                         const float *__restrict__ bias, float *logits, double *prob,
+                                                         int *topk_idx, unsigned long long *score_fx, int *natcnt,
+                                                         int *arrive, int *early_flag, int M, int N, int d, int k) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int g = lane >> 2, tg = lane & 3;
+  const int e0 = blockIdx.x * kRmExperts, t0 = blockIdx.y * kRmTokens;
+  __shared__ float s_part[8][kRmExperts * kRmTokens];
+  __shared__ int s_last;
+  const int kw = d / 8;                                   // K range of this warp: [warp*kw, warp*kw + kw)
+  const int ra = min(e0 + g, N - 1), rb = min(e0 + g + 8, N - 1);      // clamped: rows beyond N are never stored
+  const T *wa = Wr + (size_t)ra * d + warp * kw + tg * 8;
+  const T *wb = Wr + (size_t)rb * d + warp * kw + tg * 8;
+  // the router matrix is a constant of the layer: the first batch of its rows is fetched before the wait
+  uint4 A0[kRmSteps], A1[kRmSteps];
+#pragma unroll
+  for (int s = 0; s < kRmSteps; ++s) {
+    if (s * 32 < kw) {
+      A0[s] = *reinterpret_cast<const uint4 *>(wa + s * 32);
+      A1[s] = *reinterpret_cast<const uint4 *>(wb + s * 32);
+    }
+  }
+  pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  pdl_trigger();       // released only now: see router_topk_kernel
+  if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
+  const T *hb = hidden + (size_t)min(t0 + g, M - 1) * d + warp * kw + tg * 8;
+  float c[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int k0 = 0; k0 < kw; k0 += 32 * kRmSteps) {
+    uint4 Bv[kRmSteps];
+#pragma unroll
+    for (int s = 0; s < kRmSteps; ++s) {
+      if (k0 + s * 32 < kw) {
+        Bv[s] = *reinterpret_cast<const uint4 *>(hb + k0 + s * 32);
+        if (k0 > 0) {
+          A0[s] = *reinterpret_cast<const uint4 *>(wa + k0 + s * 32);
+          A1[s] = *reinterpret_cast<const uint4 *>(wb + k0 + s * 32);
+        }
+      }
+    }
+#pragma unroll
+    for (int s = 0; s < kRmSteps; ++s) {
+      if (k0 + s * 32 < kw) {
+        mma_16816(c, A0[s].x, A1[s].x, A0[s].y, A1[s].y, Bv[s].x, Bv[s].y, T());
+        mma_16816(c, A0[s].z, A1[s].z, A0[s].w, A1[s].w, Bv[s].z, Bv[s].w, T());
+      }
+    }
+  }
+  // accumulator layout: c0,c1 = (expert g, tokens 2tg, 2tg+1); c2,c3 = (expert g+8, same tokens)
+  s_part[warp][g * kRmTokens + 2 * tg] = c[0];
+  s_part[warp][g * kRmTokens + 2 * tg + 1] = c[1];
+  s_part[warp][(g + 8) * kRmTokens + 2 * tg] = c[2];
+  s_part[warp][(g + 8) * kRmTokens + 2 * tg + 1] = c[3];
+  __syncthreads();
+  if (threadIdx.x < kRmExperts * kRmTokens) {
+    const int el = threadIdx.x / kRmTokens, tl = threadIdx.x % kRmTokens;
+    float acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) acc += s_part[w][threadIdx.x];
+    if (e0 + el < N && t0 + tl < M) logits[(size_t)(t0 + tl) * N + e0 + el] = acc + (bias ? bias[e0 + el] : 0.f);
+    __threadfence();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int prev = atomicAdd(&arrive[blockIdx.y], 1);
+    s_last = (prev == (int)gridDim.x - 1);
+    if (s_last) {
+      arrive[blockIdx.y] = 0;
+      __threadfence();
+    }
+  }
+  __syncthreads();
+  if (s_last) {
+    const int t = t0 + warp;                              // eight tokens, one warp each
+    if (t < M)
+      token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane);
+  }
+}
+
+template <typename T>
+static cudaError_t launch_router_mma(const LaunchCtx &c, const void *hidden) {
+  const moespec_layer_desc &D = *c.desc;
+  const Workspace &ws = *c.ws;
+  const dim3 grid((D.n_experts + kRmExperts - 1) / kRmExperts, (c.M + kRmTokens - 1) / kRmTokens);
+  return launch_kernel(router_mma_kernel<T>, grid, dim3(256), 0, c.stream, (const T *)hidden, (const T *)D.router_w,
+                       D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.score_fx, ws.natcnt_acc, ws.arrive,
+                       ws.early_flag, c.M, D.n_experts, D.d, c.k);
+}
+template <>
+cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
+
+// Trees beyond 64 tokens of a 16-bit layer take the tensor-core router (d must split into eight K ranges of
+// whole 32-element steps).
+static bool use_router_mma(const LaunchCtx &c) {
+  static const bool off = [] { const char *v = getenv("MOESPEC_NO_ROUTER_MMA"); return v && v[0] == '1'; }();
+  return !off && is_16bit(c.desc->dtype) && c.M > 64 && c.desc->d % 256 == 0;
+}
+
 template <typename T>
 static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
+  if (use_router_mma(c)) return launch_router_mma<T>(c, hidden);
   const moespec_layer_desc &D = *c.desc;
   const Workspace &ws = *c.ws;
   const int ex_tiles = (D.n_experts + 7) / 8;
@@ -824,6 +951,8 @@ cudaError_t routing_configure() {
   set((const void *)router_topk_kernel<__half, 2>);
   set((const void *)router_topk_kernel<__half, 4>);
   set((const void *)router_topk_kernel<__half, 8>);
+  set((const void *)router_mma_kernel<__nv_bfloat16>);
+  set((const void *)router_mma_kernel<__half>);
   set((const void *)softmax_topk_kernel);
   set((const void *)route_kernel<1>);
   set((const void *)route_kernel<2>);
