@@ -578,7 +578,7 @@ int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, in
   if (e != cudaSuccess) return cuda_fail(e);
   L->last_M = M;
   L->last_k = k;
-  L->last_launches = 2;
+  L->last_launches = M > kMaxTokChunk ? 3 : 2;      // large trees add the row kernel
   return MOESPEC_OK;
 }
 

@@ -138,6 +138,18 @@ __device__ __forceinline__ void token_phase(const float *zrow, int N, int k, dou
   }
 }
 
+// Large trees leave the rows of the gather order to the row kernel (one CTA per (token, slot) pair) instead
+// of the routing kernel's last CTA, which would walk them alone.  Small trees keep them in that CTA: it is
+// faster there, and nothing waits for it.
+static bool rows_in_row_kernel(int M) { return M > kMaxTokChunk; }
+
+// In that mode the expert x token bit matrix outlives the routing kernel; the first kernel of the next call
+// clears it (every CTA takes a slice): its last readers, the row kernel's CTAs, have long finished by then.
+__device__ __forceinline__ void clear_colmask(unsigned *colmask, int words) {
+  const int cta = blockIdx.y * gridDim.x + blockIdx.x, n_cta = gridDim.x * gridDim.y;
+  for (int i = cta * blockDim.x + threadIdx.x; i < words; i += n_cta * blockDim.x) colmask[i] = 0u;
+}
+
 // ---------------------------------------------------------------------------
 // K1: z[t,i] = b_i + w_i . h_t with fp32 accumulation, fused with the token's
 // softmax and top-k.  A CTA takes TT tokens x 8 experts; warp w owns expert w of
@@ -151,8 +163,8 @@ template <typename T, int TT>
 __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                           const float *__restrict__ bias, float *logits,
                                                           double *prob, int *topk_idx, unsigned long long *score_fx,
-                                                          int *natcnt, int *arrive, int *early_flag, int M, int N,
-                                                          int d, int k) {
+                                                          int *natcnt, int *arrive, int *early_flag,
+                                                          unsigned *colmask, int M, int N, int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.y * TT;
   const int i = blockIdx.x * 8 + warp;
@@ -174,6 +186,7 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   // the call's shortlist is not known yet (the routing kernel publishes it; the FFN kernel, which can
   // only start after this kernel has finished, polls the flag)
   if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
+  clear_colmask(colmask, N * ((M + 31) >> 5));
 #ifdef MOESPEC_ROUTE_TIMING
   const long long tm0 = clock64();
 #endif
@@ -287,7 +300,8 @@ template <typename T>
 __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                          const float *__restrict__ bias, float *logits, double *prob,
                                                          int *topk_idx, unsigned long long *score_fx, int *natcnt,
-                                                         int *arrive, int *early_flag, int M, int N, int d, int k) {
+                                                         int *arrive, int *early_flag, unsigned *colmask, int M, int N,
+                                                         int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, tg = lane & 3;
   const int e0 = blockIdx.x * kRmExperts, t0 = blockIdx.y * kRmTokens;
@@ -309,6 +323,7 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
   pdl_trigger();       // released only now: see router_topk_kernel
   if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
+  clear_colmask(colmask, N * ((M + 31) >> 5));
   const T *hb = hidden + (size_t)min(t0 + g, M - 1) * d + warp * kw + tg * 8;
   float c[4] = {0.f, 0.f, 0.f, 0.f};
   for (int k0 = 0; k0 < kw; k0 += 32 * kRmSteps) {
@@ -369,7 +384,7 @@ static cudaError_t launch_router_mma(const LaunchCtx &c, const void *hidden) {
   const dim3 grid((D.n_experts + kRmExperts - 1) / kRmExperts, (c.M + kRmTokens - 1) / kRmTokens);
   return launch_kernel(router_mma_kernel<T>, grid, dim3(256), 0, c.stream, (const T *)hidden, (const T *)D.router_w,
                        D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.score_fx, ws.natcnt_acc, ws.arrive,
-                       ws.early_flag, c.M, D.n_experts, D.d, c.k);
+                       ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
 }
 template <>
 cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
@@ -378,7 +393,9 @@ cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return c
 // whole 32-element steps).
 static bool use_router_mma(const LaunchCtx &c) {
   static const bool off = [] { const char *v = getenv("MOESPEC_NO_ROUTER_MMA"); return v && v[0] == '1'; }();
-  return !off && is_16bit(c.desc->dtype) && c.M > 64 && c.desc->d % 256 == 0;
+  static const int min_m = [] { const char *v = getenv("MOESPEC_ROUTER_MMA_MIN_M"); return v ? atoi(v) : 65; }();
+  // (also for wide routers: with N >= 128 the tensor-core kernel wins at every tree size measured)
+  return !off && is_16bit(c.desc->dtype) && (c.M >= min_m || c.desc->n_experts >= 128) && c.desc->d % 256 == 0;
 }
 
 template <typename T>
@@ -397,14 +414,14 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   if (c.M <= 64 && min_tt <= 2)
     return launch_kernel(router_topk_kernel<T, 2>, dim3(ex_tiles, (c.M + 1) / 2), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
   if (c.M <= 128 && min_tt <= 4)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
   return launch_kernel(router_topk_kernel<T, 8>, dim3(ex_tiles, (c.M + 7) / 8), dim3(256), 0, c.stream,
                        (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                       ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, c.M, D.n_experts, D.d, c.k);
+                       ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
@@ -416,11 +433,12 @@ cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
 // Softmax and top-k from caller-supplied logits: one warp per token.
 __global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, double *prob, int *topk_idx,
                                                            unsigned long long *score_fx, int *natcnt, int *early_flag,
-                                                           int M, int N, int k) {
+                                                           unsigned *colmask, int M, int N, int k) {
   const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
   pdl_trigger();
   pdl_wait();
   if (early_flag && blockIdx.x == 0 && threadIdx.x == 0) *early_flag = 0;
+  clear_colmask(colmask, N * ((M + 31) >> 5));
   if (t < M)
     token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt,
                 threadIdx.x & 31);
@@ -448,6 +466,7 @@ struct RouteArgs {
   long long expert_bytes;       // 3*d*f*sizeof(dtype)
   int early;                    // the FFN kernel starts on the shortlist before this kernel has finished
   int ffn_ctas;                 // CTAs of the FFN kernel: CTA c starts on gate/up unit c of the list
+  int rows_later;               // the row of every (token, slot) pair is left to the row kernel (large trees)
 };
 
 constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
@@ -738,7 +757,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   //   warps 0-3  row of every (token, slot)       warps 4-6  work-unit list       warp 7  coverage
   const int n_chunks = a.early ? s_nchunks : s_unit_base[N];
   double cov = 0.0;
-  if (warp < 4) {
+  if (warp < 4 && !a.rows_later) {
     // rows ordered by (expert ascending, token ascending): the row of (t, e) is
     // offset[e] + number of tokens below t that were also routed to e
     // thread -> (token, slot) with the slot count padded to a power of two (no integer division)
@@ -775,7 +794,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         ws.tokslot2row[(size_t)tt * k + slot] = row;
       }
     }
-  } else if (warp < 7) {
+  } else if (warp >= 4 && warp < 7) {
     // tensor-core work units (expert, token chunk, 128-row slab): all gate/up units, then all down
     // units, each group ordered by (expert, chunk, slab); ready counters and the dispenser start at 0
     if (a.tiles_up > 0) {
@@ -813,7 +832,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         ws.units[u] = Unit{e, tl, row0, rows, s_unit_base[e] + c, phase, 0, 0};
       }
     }
-  } else {
+  } else if (warp == 7) {
     for (int r = lane; r < nS; r += 32) cov += (double)s_fx[s_Srank[r]];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cov += shfl_xor_double(cov, o);
@@ -856,7 +875,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     ws.natcnt_acc[i] = 0;
     ws.count_acc[i] = 0;
   }
-  for (int i = tid; i < N * used_words; i += blockDim.x) ws.colmask[i] = 0u;
+  // with rows_later the bit matrix is still needed by the row kernel and is cleared by the next call's
+  // first kernel instead
+  if (!a.rows_later)
+    for (int i = tid; i < N * used_words; i += blockDim.x) ws.colmask[i] = 0u;
 }
 
 static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) {
@@ -871,6 +893,7 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.expert_bytes = 3LL * D.d * D.f * dtype_bytes(D.dtype);
   a.early = c.ru > 0 ? c.early : 0;
   a.ffn_ctas = tc_grid_size(D.device);
+  a.rows_later = rows_in_row_kernel(c.M);
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
   if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);
@@ -902,14 +925,16 @@ cudaError_t launch_route_after_router(const LaunchCtx &c) { return launch_route_
 // Routing from caller-supplied logits: per-token softmax/top-k first (two launches).
 cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
   cudaError_t e = launch_kernel(softmax_topk_kernel, dim3((c.M + 3) / 4), dim3(128), 0, c.stream, logits, c.ws->prob,
-                                c.ws->topk_idx, c.ws->score_fx, c.ws->natcnt_acc, c.ws->early_flag, c.M, c.desc->n_experts,
-                                c.k);
+                                c.ws->topk_idx, c.ws->score_fx, c.ws->natcnt_acc, c.ws->early_flag, c.ws->colmask, c.M,
+                                c.desc->n_experts, c.k);
   if (e != cudaSuccess) return e;
-  return launch_route_kernel(c, logits);
+  e = launch_route_kernel(c, logits);
+  if (e != cudaSuccess || !rows_in_row_kernel(c.M)) return e;
+  return launch_gather(c, nullptr);       // rows only: there is no hidden state on this path
 }
 
 // ---------------------------------------------------------------------------
-// K3: gather routed rows: x_perm[r, :] = hidden[perm_row2tok[r], :].
+// K3: gather routed rows: x_perm[r, :] = hidden[perm_row2tok[r], :] (Appendix C), one CTA per row.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restrict__ hidden,
                                                           uint4 *__restrict__ x_perm,
@@ -925,13 +950,63 @@ __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restric
   for (int j = threadIdx.x; j < row_vec; j += blockDim.x) dst[j] = src[j];
 }
 
+// The same for large trees, where the rows themselves are still to be worked out: one CTA per (token, slot)
+// pair.  Rows are ordered by (expert ascending, token ascending): the row of (t, e) is offset[e] + the
+// number of tokens below t that were also routed to e, a popcount prefix over expert e's row of the bit
+// matrix.  The CTA records the row in both directions and, when `hidden` is given, copies the token's
+// hidden state there.
+__global__ void __launch_bounds__(128) rows_gather_kernel(const uint4 *__restrict__ hidden, uint4 *__restrict__ x_perm,
+                                                          const int *__restrict__ assign_idx,
+                                                          const int *__restrict__ offset,
+                                                          const unsigned *__restrict__ colmask, int *perm_row2tok,
+                                                          int *row2expert, int *tokslot2row, int M, int k,
+                                                          int row_vec) {
+  const int pair = blockIdx.x, t = pair / k;
+  const int lane = threadIdx.x & 31;
+  __shared__ int s_row;
+  pdl_trigger();
+  pdl_wait();
+  const int e = assign_idx[pair];
+  if (e < 0) {                                  // dropped slot (truncation, or fewer than k experts kept)
+    if (threadIdx.x == 0) tokslot2row[pair] = -1;
+    return;
+  }
+  if (threadIdx.x < 32) {
+    const unsigned *cm = colmask + (size_t)e * ((M + 31) >> 5);
+    const int full = t >> 5;
+    int below = 0;
+    for (int w = lane; w < full; w += 32) below += __popc(cm[w]);
+    if (lane == 0) below += __popc(cm[full] & ((1u << (t & 31)) - 1u));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(kFull, below, o);
+    if (lane == 0) {
+      const int row = offset[e] + below;
+      s_row = row;
+      perm_row2tok[row] = t;
+      if (row2expert) row2expert[row] = e;
+      tokslot2row[pair] = row;
+    }
+  }
+  if (!hidden) return;
+  __syncthreads();
+  const uint4 *src = hidden + (size_t)t * row_vec;
+  uint4 *dst = x_perm + (size_t)s_row * row_vec;
+  for (int j = threadIdx.x; j < row_vec; j += blockDim.x) dst[j] = src[j];
+}
+
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
   const moespec_layer_desc &D = *c.desc;
+  const Workspace &ws = *c.ws;
   const int row_vec = D.d * dtype_bytes(D.dtype) / 16;
   const int rows = c.M * c.k;
   if (rows == 0) return cudaSuccess;
+  if (rows_in_row_kernel(c.M))
+    return launch_kernel(rows_gather_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,
+                         (uint4 *)ws.x_perm, (const int *)ws.assign_idx, (const int *)ws.offset,
+                         (const unsigned *)ws.colmask, ws.perm_row2tok, ws.row2expert, ws.tokslot2row, c.M, c.k,
+                         row_vec);
   return launch_kernel(gather_rows_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,
-                       (uint4 *)c.ws->x_perm, (const int *)c.ws->perm_row2tok, (const int *)c.ws->counters, row_vec);
+                       (uint4 *)ws.x_perm, (const int *)ws.perm_row2tok, (const int *)ws.counters, row_vec);
 }
 
 // The FFN kernel needs nearly all of an SM's shared memory.  An SM whose L1/shared split was chosen for
@@ -959,6 +1034,7 @@ cudaError_t routing_configure() {
   set((const void *)route_kernel<4>);
   set((const void *)route_kernel<8>);
   set((const void *)gather_rows_kernel);
+  set((const void *)rows_gather_kernel);
   return e;
 }
 
