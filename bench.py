@@ -309,6 +309,10 @@ def run_tables(args, device):
         L = cfg.n_layers
         n_copies = L if L > 1 else (2 if name == "mixtral" else 4)
         Ms, Bs = synth.SWEEPS[name]["M"], synth.SWEEPS[name]["B"]
+        if args.only_M:          # one point (or a few) instead of the sweep, e.g. for a profiler capture
+            Ms = [int(x) for x in args.only_M.split(",")]
+        if args.only_B:
+            Bs = [int(x) for x in args.only_B.split(",")]
         max_M = max(Ms)
         weights = [synth.gen_layer(cfg, seed=2000, layer=l, device=device) for l in range(n_copies)]
         out_dtype = torch.bfloat16 if L > 1 else torch.float32
@@ -437,6 +441,8 @@ def main():
                     "of each and print one JSON line per point instead of the benchmark line")
     ap.add_argument("--tables-cpu", action="store_true",
                     help="with --tables: also time the CPU oracle once per point (one layer, host cores)")
+    ap.add_argument("--only-M", default="", help="with --tables: tree sizes to run instead of the workload's sweep")
+    ap.add_argument("--only-B", default="", help="with --tables: budgets to run instead of the workload's sweep")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed steps (for profiler captures); prints a short line")
     args = ap.parse_args()
