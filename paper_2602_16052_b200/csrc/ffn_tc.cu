@@ -6,7 +6,7 @@
 // (small budgets, small trees): an SM can only stream ~55-100 GB/s, so HBM is
 // only saturated when every SM has work.  Weights are the MMA A operand (rows of
 // W on the M axis; the MMA is always M = 128 and rows beyond RU are ignored),
-// routed token rows are the B operand (N axis, padded to a multiple of 32),
+// routed token rows are the B operand (N axis, padded to 16 or a multiple of 32),
 // fp32 accumulators live in tensor memory (two buffers, so the epilogue of one
 // unit overlaps the MMAs of the next).
 //
@@ -23,7 +23,16 @@
 // Units are handed out in order and gate/up units never wait, so every unit a
 // down unit waits for is already running or done: there is no circular wait.
 //
-// Six warps per CTA:
+// Early start (trees of up to 128 tokens): the CTAs of this kernel are resident
+// while the routing kernels still run.  CTA c does not wait for them: as soon as
+// the routing kernel has published the shortlist (a flag; at once when the
+// shortlist is fixed) it starts on gate/up unit c of the rank-ordered list --
+// expert S_rank[c / slabs], slab c % slabs -- with ALL tokens of the tree as the
+// B operand, read from `hidden` itself, and keeps the routed tokens' columns in
+// the epilogue, by which time the gather order exists.  The routing kernel lists
+// the units in the same order, so unit c of the list is that unit.
+//
+// Ten warps per CTA:
 //   warp 0        : dispenser + TMA producer.  Lane 0 waits and draws units; all
 //                   lanes issue the copies of a stage: 64-wide K chunks of the
 //                   weight slab(s) (3-D tensor map, expert id is the outer
@@ -36,9 +45,9 @@
 //                   shared by two warps, which take alternate groups of 16
 //                   columns), apply SwiGLU, store to global.
 // The combine of the layer lives in this kernel too: after its last unit every
-// CTA waits (bounded) until all down units are stored and then produces its share
-// of `out` from y, the mixing weights and tokslot2row, adding slots in a fixed
-// order.  (Fetching routed rows straight from `hidden` with one-row TMA boxes was
+// CTA waits (bounded) until all down units are stored and then its warps produce
+// their share of `out` from y, the mixing weights and tokslot2row (128 columns of
+// one token per warp and step), adding slots in a fixed order.  (Fetching routed rows straight from `hidden` with one-row TMA boxes was
 // measured 40 % slower than reading a gathered copy with 32-row boxes: the copy
 // engine's rate for 128-byte boxes is the limit.)
 // Every wait is bounded: on expiry the CTA raises an abort flag, records

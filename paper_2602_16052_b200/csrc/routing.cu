@@ -4,15 +4,19 @@
 // truncation (Eq. 7) with the mixing weights of Section 3.3, and the
 // per-expert gather order (Appendix C).
 //
-// Two launches:
+// Three launches:
 //   router_topk_kernel   router dot products; the CTA that finishes a token
 //                        tile's last logit also runs those tokens' softmax and
 //                        top-k and adds their probabilities to the per-expert
-//                        scores (a counter, never a wait)
+//                        scores (a counter, never a wait).  router_mma_kernel is
+//                        the same on the tensor cores, for larger trees.
 //   route_kernel         eight tokens per CTA: every CTA ranks the scores itself
-//                        (shortlist), re-routes its tokens, and the CTA that
-//                        finishes last does the scan, the gather order, the
-//                        work-unit list and the statistics
+//                        (shortlist; CTA 0 publishes it for the FFN kernel),
+//                        re-routes its tokens, and the CTA that finishes last
+//                        does the scan, the gather order, the work-unit list and
+//                        the statistics
+//   gather_rows_kernel   x_perm[row] = hidden[token] (rows_gather_kernel also
+//                        works out the rows, for trees above 128 tokens)
 // Scores are accumulated as 2^-52 fixed-point integers, so the sum does not
 // depend on the order in which tokens arrive and identical experts tie exactly.
 // A stand-alone softmax/top-k kernel serves callers that inject logits.
