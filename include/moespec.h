@@ -110,6 +110,10 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
  * aligned.  out: device [M, d] in out_dtype, fully overwritten (exact zeros for a token with
  * no kept expert when residual = 0).  out must not alias hidden.
  * stream: a cudaStream_t (NULL = default stream).  Enqueues and returns.
+ * A handle owns one workspace: calls on the same handle must be ordered (same
+ * stream, or synchronised by the caller); different handles are independent.
+ * The call may be captured into a CUDA graph by the caller (it allocates nothing
+ * and only enqueues kernels).
  * Errors: BAD_HANDLE, NULL_POINTER, INVALID_ARG, CUDA (launch failure). */
 int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int k, int B,
                          void *out, void *stream);
