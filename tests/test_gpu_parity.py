@@ -317,6 +317,31 @@ def test_repeat_calls_are_bitwise_reproducible():
     layer.destroy()
 
 
+def test_device_entry_can_be_captured_into_a_callers_graph():
+    """moespec_verify_layer allocates nothing and only enqueues kernels: a caller may capture it into its own
+    CUDA graph and replay it; replays give the bits of a direct call, also after the input has changed."""
+    cfg = synth.CONFIGS["olmoe"].with_(f=256)
+    case = H.make_case(cfg, 63, seed=33)
+    layer = make_layer(case, 63, cfg.k, out_dtype=torch.float32)
+    x = case["hidden"].clone()
+    out = torch.empty((63, cfg.d), dtype=torch.float32, device="cuda")
+    layer.verify_layer(x, cfg.k, 16, out)                     # warm-up outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        layer.verify_layer(x, cfg.k, 16, out)
+    for seed in (33, 34):
+        x.copy_(synth.gen_hidden(cfg, 63, seed=seed, device="cuda"))
+        g.replay()
+        torch.cuda.synchronize()
+        replayed = out.clone()
+        direct = layer.verify_layer(x, cfg.k, 16).clone()
+        torch.cuda.synchronize()
+        assert torch.equal(replayed, direct)
+        assert layer.get_stats()["status"] == 0
+    layer.destroy()
+
+
 # ------------------------------------------------------------------ argument errors (host side only)
 def test_argument_errors_return_codes():
     m = ms()
