@@ -88,6 +88,25 @@ def test_stack_per_layer_parity_with_per_layer_budgets(policy_name, mode_name, r
         layer.destroy()
 
 
+def test_stack_at_full_layer_size():
+    """Four layers of the 16-layer benchmark stack at their full size (d=2048, N=64, f=1024, M=63, B=32), in
+    the configuration the benchmark times (one graph launch, bf16 residual stream), each layer checked
+    against the oracle on the GPU's own input to that layer."""
+    cfg = synth.CONFIGS["olmoe16"].with_(n_layers=4)
+    M, B = 63, 32
+    cases, layers, stack = build_stack(cfg, M, seed=2000)
+    x0 = synth.gen_hidden(cfg, M, seed=2000, device="cuda")
+    out = stack.verify_stack(x0, cfg.k, B)
+    torch.cuda.synchronize()
+    xs = [x0.cpu()] + [stack.get_stream(l) for l in range(1, cfg.n_layers)] + [out.cpu()]
+    check_layers(cfg, cases, layers, xs, [B] * cfg.n_layers, orc.SUBSTITUTION, orc.FROM_ALL, True)
+    for layer in layers:
+        assert layer.get_stats()["n_active"] == B
+    stack.destroy()
+    for layer in layers:
+        layer.destroy()
+
+
 def test_stack_host_entry_and_static_ranking_change():
     m = ms()
     cfg = synth.CONFIGS["olmoe"].with_(f=128, n_experts=16, n_layers=3)
