@@ -355,6 +355,7 @@ int moespec_reconstruction_error(moespec_layer_t *layer, const void *out_S, cons
 const char *moespec_strerror(int status);
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int moespec_last_cuda_error(void);
+/* major*100 + minor; 110 added the stack, the analysis mode and the early-start FFN kernel. */
 int moespec_version(void);
 
 #ifdef __cplusplus

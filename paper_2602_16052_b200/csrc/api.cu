@@ -737,7 +737,7 @@ const char *moespec_strerror(int status) {
 }
 
 int moespec_last_cuda_error(void) { return tl_cuda_error; }
-int moespec_version(void) { return 100; }
+int moespec_version(void) { return 110; }
 
 }  // extern "C"
 
