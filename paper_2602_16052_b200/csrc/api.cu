@@ -11,6 +11,16 @@
 using namespace moespec;
 
 constexpr int kMaxProfiled = 8;   // kernels per verify call that can be bracketed by events
+constexpr int kGraphCache = 4;    // instantiated graphs kept per handle (least recently used is replaced)
+
+// One cached instantiation of the host entry point: the step for (M, k, B, buffer pair).
+struct HostGraph {
+  cudaGraphExec_t exec = nullptr;
+  int M = 0, k = 0, B = 0;
+  const void *in = nullptr;
+  void *out = nullptr;
+  unsigned long long used = 0;
+};
 
 struct moespec_layer {
   unsigned long long magic;
@@ -28,10 +38,8 @@ struct moespec_layer {
   // host-buffer entry point: the copy-in, the kernels and the copy-out as one instantiated graph
   cudaStream_t own_stream;
   cudaEvent_t ev_in;
-  cudaGraphExec_t host_exec;
-  int hg_M, hg_k, hg_B;
-  const void *hg_in;
-  void *hg_out;
+  HostGraph host_graph[kGraphCache];
+  unsigned long long graph_clock;
   bool graph_usable;
   long long debug_spin_limit;
   int debug_ready_bias;
@@ -54,13 +62,17 @@ struct moespec_stack {
   bool graph_on, graph_usable;
   cudaStream_t own_stream;
   cudaEvent_t ev_in;
-  cudaGraphExec_t exec;     // one cached instantiation: (M, k, budgets, buffers, epochs)
-  int g_M, g_k;
-  std::vector<int> g_B;
-  const void *g_in;
-  void *g_out;
-  bool g_host;
-  unsigned g_epoch;
+  struct Graph {            // one cached instantiation: (M, k, budgets, buffers, epochs)
+    cudaGraphExec_t exec = nullptr;
+    int M = 0, k = 0;
+    std::vector<int> B;
+    const void *in = nullptr;
+    void *out = nullptr;
+    bool host = false;
+    unsigned epoch = 0;
+    unsigned long long used = 0;
+  } graph[kGraphCache];
+  unsigned long long graph_clock;
   int last_M, last_launches;
 };
 
@@ -77,6 +89,12 @@ int cuda_fail(cudaError_t e) {
   tl_cuda_error = (int)e;
   return e == cudaErrorMemoryAllocation ? MOESPEC_ERR_OUT_OF_MEMORY : MOESPEC_ERR_CUDA;
 }
+
+}  // namespace
+namespace moespec {
+void record_cuda_error(cudaError_t e) { tl_cuda_error = (int)e; }
+}
+namespace {
 
 bool is_live(moespec_layer *L) {
   if (!L) return false;
@@ -105,6 +123,14 @@ struct DeviceGuard {
     if (changed) cudaSetDevice(prev);
   }
 };
+
+// A captured graph has the layer's settings baked into its kernel arguments: drop them all.
+void drop_host_graphs(moespec_layer *L) {
+  for (HostGraph &g : L->host_graph) {
+    if (g.exec) cudaGraphExecDestroy(g.exec);
+    g = HostGraph();
+  }
+}
 
 size_t elt_bytes(const moespec_layer_desc &d) { return dtype_bytes(d.dtype); }
 size_t out_elt_bytes(const moespec_layer_desc &d) { return dtype_bytes(d.out_dtype ? d.out_dtype : d.dtype); }
@@ -185,7 +211,7 @@ int validate_call(moespec_layer *L, int M, int k, int B) {
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 bool zero_copy_enabled() {
-  static const bool off = [] { const char *v = getenv("MOESPEC_NO_ZERO_COPY"); return v && v[0] == '1'; }();
+  static const bool off = [] { const char *v = experiment_env("MOESPEC_NO_ZERO_COPY"); return v && v[0] == '1'; }();
   return !off;
 }
 
@@ -271,7 +297,7 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
 namespace moespec {
 bool pdl_enabled() {
   static const bool on = [] {
-    const char *v = getenv("MOESPEC_NO_PDL");
+    const char *v = experiment_env("MOESPEC_NO_PDL");
     return !(v && v[0] == '1');
   }();
   return on;
@@ -336,6 +362,16 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
     return cuda_fail(e);
   }
   carve(d, L->R_cap, static_cast<char *>(L->arena), &L->ws);
+  if (!use_tc) {
+    // the CUDA-core FFN stages a row of d (gate/up) or f (down) floats in shared memory
+    bool fits = true;
+    e = cc_configure(d, &fits);
+    if (e != cudaSuccess || !fits) {
+      cudaFree(L->arena);
+      delete L;
+      return e != cudaSuccess ? cuda_fail(e) : MOESPEC_ERR_UNSUPPORTED;
+    }
+  }
   if (use_tc) {
     int cu_res = 0;
     e = tc_encode_maps(d, L->ws, L->R_cap, &L->maps, &cu_res);
@@ -354,7 +390,7 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   L->epoch = 0;
   L->analysis = nullptr;
   L->an_M = L->an_k = 0;
-  L->host_exec = nullptr;
+  L->graph_clock = 0;
   L->graph_usable = cudaStreamCreateWithFlags(&L->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&L->ev_in, cudaEventDisableTiming) == cudaSuccess;
   for (int i = 0; i <= kMaxProfiled; ++i) {
@@ -410,13 +446,18 @@ int moespec_verify_layer_host(moespec_layer_t *L, const void *hidden_host, int M
   const bool zero_copy = in_dev && out_dev && aligned16(in_dev) && aligned16(out_dev) && bytes % 16 == 0 &&
                          zero_copy_enabled();
   if (L->graph_usable && !L->profiling && is_pinned(hidden_host) && is_pinned(out_host)) {
-    const bool hit = L->host_exec && L->hg_M == M && L->hg_k == k && L->hg_B == B && L->hg_in == hidden_host &&
-                     L->hg_out == out_host;
+    // a few instantiations are kept (a caller may alternate between trees or buffer pairs); a miss replaces
+    // the least recently used one
+    HostGraph *slot = nullptr;
+    for (HostGraph &g : L->host_graph)
+      if (g.exec && g.M == M && g.k == k && g.B == B && g.in == hidden_host && g.out == out_host) slot = &g;
+    const bool hit = slot != nullptr;
     if (!hit) {
-      if (L->host_exec) {
-        cudaGraphExecDestroy(L->host_exec);
-        L->host_exec = nullptr;
-      }
+      slot = &L->host_graph[0];
+      for (HostGraph &g : L->host_graph)
+        if (!g.exec || (slot->exec && g.used < slot->used)) slot = &g;
+      if (slot->exec) cudaGraphExecDestroy(slot->exec);
+      *slot = HostGraph();
       cudaGraph_t graph = nullptr;
       e = cudaStreamBeginCapture(L->own_stream, cudaStreamCaptureModeThreadLocal);
       if (e == cudaSuccess) {
@@ -437,22 +478,23 @@ int moespec_verify_layer_host(moespec_layer_t *L, const void *hidden_host, int M
         cudaError_t e2 = cudaStreamEndCapture(L->own_stream, &graph);
         if (e == cudaSuccess) e = e2;
       }
-      if (e == cudaSuccess) e = cudaGraphInstantiate(&L->host_exec, graph, 0);
+      if (e == cudaSuccess) e = cudaGraphInstantiate(&slot->exec, graph, 0);
       if (graph) cudaGraphDestroy(graph);
       if (e != cudaSuccess) {          // graphs unavailable here: use the plain path from now on
         cudaGetLastError();
-        L->host_exec = nullptr;
+        slot->exec = nullptr;
         L->graph_usable = false;
       } else {
-        L->hg_M = M; L->hg_k = k; L->hg_B = B; L->hg_in = hidden_host; L->hg_out = out_host;
+        slot->M = M; slot->k = k; slot->B = B; slot->in = hidden_host; slot->out = out_host;
       }
     }
-    if (L->host_exec) {
+    if (slot->exec) {
+      slot->used = ++L->graph_clock;
       // work already queued on the caller's stream (e.g. a weight update) is waited for first; the replay
       // itself runs on the internal stream (measured faster than replaying on the legacy default stream)
       if ((e = cudaEventRecord(L->ev_in, s)) != cudaSuccess) return cuda_fail(e);
       if ((e = cudaStreamWaitEvent(L->own_stream, L->ev_in, 0)) != cudaSuccess) return cuda_fail(e);
-      if ((e = cudaGraphLaunch(L->host_exec, L->own_stream)) != cudaSuccess) return cuda_fail(e);
+      if ((e = cudaGraphLaunch(slot->exec, L->own_stream)) != cudaSuccess) return cuda_fail(e);
       if ((e = cudaStreamSynchronize(L->own_stream)) != cudaSuccess) return cuda_fail(e);
       return MOESPEC_OK;
     }
@@ -556,10 +598,7 @@ int moespec_set_static_ranking(moespec_layer_t *L, const int *ranked_host, int n
   if (e != cudaSuccess) return cuda_fail(e);
   L->ws.n_static = (int)order.size();
   ++L->epoch;
-  if (L->host_exec) {            // a captured graph has the old ordering size baked into its arguments
-    cudaGraphExecDestroy(L->host_exec);
-    L->host_exec = nullptr;
-  }
+  drop_host_graphs(L);           // a captured graph has the old ordering size baked into its arguments
   return MOESPEC_OK;
 }
 
@@ -660,10 +699,7 @@ int moespec_debug_set_wait(moespec_layer_t *L, long long limit_cycles, int ready
   L->debug_spin_limit = limit_cycles;
   L->debug_ready_bias = ready_bias;
   ++L->epoch;
-  if (L->host_exec) {            // a captured graph has the old values baked in
-    cudaGraphExecDestroy(L->host_exec);
-    L->host_exec = nullptr;
-  }
+  drop_host_graphs(L);           // a captured graph has the old values baked in
   return MOESPEC_OK;
 }
 
@@ -706,7 +742,7 @@ int moespec_destroy(moespec_layer_t *L) {
   {
     DeviceGuard guard(L->desc.device);
     for (int i = 0; i <= kMaxProfiled; ++i) cudaEventDestroy(L->ev[i]);
-    if (L->host_exec) cudaGraphExecDestroy(L->host_exec);
+    drop_host_graphs(L);
     if (L->graph_usable) {
       cudaEventDestroy(L->ev_in);
       cudaStreamDestroy(L->own_stream);
@@ -793,13 +829,23 @@ int stack_validate(moespec_stack *S, int M, int k, const int *B) {
 cudaGraphExec_t stack_graph(moespec_stack *S, const void *in, int M, int k, const int *B, void *out, bool host) {
   const int L = (int)S->layers.size();
   const unsigned epoch = stack_epoch(S);
-  bool hit = S->exec && S->g_M == M && S->g_k == k && S->g_in == in && S->g_out == out && S->g_host == host &&
-             S->g_epoch == epoch;
-  for (int l = 0; hit && l < L; ++l) hit = S->g_B[l] == B[l];
-  if (hit) return S->exec;
-  if (S->exec) {
-    cudaGraphExecDestroy(S->exec);
-    S->exec = nullptr;
+  for (moespec_stack::Graph &g : S->graph) {
+    bool hit = g.exec && g.M == M && g.k == k && g.in == in && g.out == out && g.host == host && g.epoch == epoch;
+    for (int l = 0; hit && l < L; ++l) hit = g.B[l] == B[l];
+    if (hit) {
+      g.used = ++S->graph_clock;
+      return g.exec;
+    }
+  }
+  // miss: replace an instantiation whose layer settings are stale, else the least recently used one
+  moespec_stack::Graph *slot = &S->graph[0];
+  for (moespec_stack::Graph &g : S->graph) {
+    const bool g_dead = !g.exec || g.epoch != epoch, s_dead = !slot->exec || slot->epoch != epoch;
+    if ((g_dead && !s_dead) || (g_dead == s_dead && g.used < slot->used)) slot = &g;
+  }
+  if (slot->exec) {
+    cudaGraphExecDestroy(slot->exec);
+    slot->exec = nullptr;
   }
   const size_t bytes = (size_t)M * S->row_bytes;
   const void *dev_in = host ? S->in_stage : in;
@@ -826,17 +872,18 @@ cudaGraphExec_t stack_graph(moespec_stack *S, const void *in, int M, int k, cons
     cudaError_t e2 = cudaStreamEndCapture(S->own_stream, &graph);
     if (e == cudaSuccess) e = e2;
   }
-  if (e == cudaSuccess) e = cudaGraphInstantiate(&S->exec, graph, 0);
+  if (e == cudaSuccess) e = cudaGraphInstantiate(&slot->exec, graph, 0);
   if (graph) cudaGraphDestroy(graph);
   if (e != cudaSuccess) {
     cudaGetLastError();
-    S->exec = nullptr;
+    slot->exec = nullptr;
     S->graph_usable = false;
     return nullptr;
   }
-  S->g_M = M; S->g_k = k; S->g_in = in; S->g_out = out; S->g_host = host; S->g_epoch = epoch;
-  S->g_B.assign(B, B + L);
-  return S->exec;
+  slot->M = M; slot->k = k; slot->in = in; slot->out = out; slot->host = host; slot->epoch = epoch;
+  slot->B.assign(B, B + L);
+  slot->used = ++S->graph_clock;
+  return slot->exec;
 }
 
 }  // namespace
@@ -883,7 +930,7 @@ int moespec_stack_create(moespec_layer_t *const *layers, int n_layers, moespec_s
   S->arena = static_cast<char *>(p);
   S->in_stage = S->arena + slab * (size_t)(n_layers - 1);
   S->out_stage = S->in_stage + slab;
-  S->exec = nullptr;
+  S->graph_clock = 0;
   S->graph_on = true;
   S->graph_usable = cudaStreamCreateWithFlags(&S->own_stream, cudaStreamNonBlocking) == cudaSuccess &&
                     cudaEventCreateWithFlags(&S->ev_in, cudaEventDisableTiming) == cudaSuccess;
@@ -985,7 +1032,8 @@ int moespec_stack_destroy(moespec_stack_t *S) {
   int rc = MOESPEC_OK;
   {
     DeviceGuard guard(S->device);
-    if (S->exec) cudaGraphExecDestroy(S->exec);
+    for (moespec_stack::Graph &g : S->graph)
+      if (g.exec) cudaGraphExecDestroy(g.exec);
     if (S->graph_usable) {
       cudaEventDestroy(S->ev_in);
       cudaStreamDestroy(S->own_stream);

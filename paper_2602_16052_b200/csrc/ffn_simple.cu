@@ -110,6 +110,30 @@ static cudaError_t launch_cc(const LaunchCtx &c, int phase) {
   }
 }
 
+// The kernels stage one row (d or f floats) in dynamic shared memory; rows beyond 48 KB need the opt-in
+// limit raised, and rows beyond the device's opt-in maximum do not fit at all (*fits = false).
+template <typename T>
+static cudaError_t configure_cc(size_t up_bytes, size_t down_bytes) {
+  cudaError_t e = cudaSuccess;
+  if (up_bytes > 48 * 1024)
+    e = cudaFuncSetAttribute(ffn_gateup_cc_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)up_bytes);
+  if (e == cudaSuccess && down_bytes > 48 * 1024)
+    e = cudaFuncSetAttribute(ffn_down_cc_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)down_bytes);
+  return e;
+}
+
+cudaError_t cc_configure(const moespec_layer_desc &D, bool *fits) {
+  const size_t up_bytes = (size_t)D.d * sizeof(float), down_bytes = (size_t)D.f * sizeof(float);
+  int optin = 0;
+  cudaError_t e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, D.device);
+  if (e != cudaSuccess) return e;
+  *fits = up_bytes <= (size_t)optin && down_bytes <= (size_t)optin;
+  if (!*fits) return cudaSuccess;
+  if (D.dtype == MOESPEC_BF16) return configure_cc<__nv_bfloat16>(up_bytes, down_bytes);
+  if (D.dtype == MOESPEC_FP16) return configure_cc<__half>(up_bytes, down_bytes);
+  return configure_cc<float>(up_bytes, down_bytes);
+}
+
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase) {
   if (c.desc->dtype == MOESPEC_BF16) return launch_cc<__nv_bfloat16>(c, phase);
   if (c.desc->dtype == MOESPEC_FP16) return launch_cc<__half>(c, phase);

@@ -817,7 +817,7 @@ cudaError_t tc_configure() {
 
 // Early start needs every token in one MMA (N <= 128) and is an option of the tensor-core path.
 bool tc_early_start(const moespec_layer_desc &d, int M) {
-  static const bool off = [] { const char *v = getenv("MOESPEC_NO_EARLY"); return v && v[0] == '1'; }();
+  static const bool off = [] { const char *v = experiment_env("MOESPEC_NO_EARLY"); return v && v[0] == '1'; }();
   return !off && is_16bit(d.dtype) && M >= 1 && M <= kMaxTokChunk;
 }
 
@@ -838,7 +838,7 @@ int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
   // otherwise be fewer gate/up units than half the SMs (a handful of kept experts, e.g. M = 1).
   int active = B < D.n_experts ? B : D.n_experts;          // upper bound of kept experts that get rows
   if ((long long)M * k < active) active = M * k;
-  static const int forced = [] { const char *v = getenv("MOESPEC_FORCE_RU"); return v ? atoi(v) : 0; }();
+  static const int forced = [] { const char *v = experiment_env("MOESPEC_FORCE_RU"); return v ? atoi(v) : 0; }();
   if (forced == 128 || forced == 64 || forced == 32) return forced;     // experiments only
   return (long long)active * (D.f / kTile) * 2 < sm_count_cached(D.device) ? 64 : kTile;
 }
@@ -846,7 +846,7 @@ int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
 // Down units use 128-row slabs: half-height ones would shorten the tail of the list but double the copies
 // per stage, and measured 10 % slower overall.
 int tc_rows_per_down_unit(int ru) {
-  static const int forced = [] { const char *v = getenv("MOESPEC_FORCE_RU_DOWN"); return v ? atoi(v) : 0; }();
+  static const int forced = [] { const char *v = experiment_env("MOESPEC_FORCE_RU_DOWN"); return v ? atoi(v) : 0; }();
   if (forced == 128 || forced == 64 || forced == 32) return forced;     // experiments only
   (void)ru;
   return kTile;

@@ -5,9 +5,22 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include "../../include/moespec.h"
 
 namespace moespec {
+
+// Switches that choose between equivalent code paths (for A/B measurements) are read from the
+// environment only in builds made with -DMOESPEC_EXPERIMENTS; the shipped library reads no
+// behaviour from the environment.
+#ifdef MOESPEC_EXPERIMENTS
+inline const char *experiment_env(const char *name) { return getenv(name); }
+#else
+inline const char *experiment_env(const char *) { return nullptr; }
+#endif
+
+// Remember the cudaError_t of a failing call for moespec_last_cuda_error() (per thread).
+void record_cuda_error(cudaError_t e);
 
 inline bool is_16bit(int dtype) { return dtype == MOESPEC_BF16 || dtype == MOESPEC_FP16; }
 inline int dtype_bytes(int dtype) { return is_16bit(dtype) ? 2 : 4; }
@@ -97,7 +110,7 @@ struct LaunchCtx {
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
-bool pdl_enabled();   // false when MOESPEC_NO_PDL=1 is set in the environment
+bool pdl_enabled();   // true (an experiments build can switch programmatic launches off)
 
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
@@ -124,6 +137,7 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden);
 cudaError_t routing_configure();   // one-time function attributes of the routing kernels (tensor-core path)
 // ffn_simple.cu
 cudaError_t launch_ffn_cuda_core(const LaunchCtx &c, int phase);   // 0 gate/up, 1 down
+cudaError_t cc_configure(const moespec_layer_desc &d, bool *fits);   // shared-memory opt-in of the CUDA-core FFN
 // ffn_tc.cu
 struct TcMaps {            // per handle: weight maps for slab heights 128, 64, 32
   CUtensorMap w_gate[3], w_up[3], w_down[3];

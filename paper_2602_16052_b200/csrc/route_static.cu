@@ -86,8 +86,14 @@ extern "C" int moespec_route_static(const float *logits, int M, int N, int k, in
       !tokslot2row || !score || !summary)
     return MOESPEC_ERR_NULL_POINTER;
 
+  // a failing CUDA call is remembered for moespec_last_cuda_error(), as in the handle-based entry points
+  auto cuda_fail = [](cudaError_t e) {
+    record_cuda_error(e);
+    return (int)MOESPEC_ERR_CUDA;
+  };
   unsigned char *scratch = nullptr;
-  if (scratch_for_current_device(&scratch) != cudaSuccess) return MOESPEC_ERR_CUDA;
+  cudaError_t e = scratch_for_current_device(&scratch);
+  if (e != cudaSuccess) return cuda_fail(e);
 
   Workspace ws{};
   ws.prob = reinterpret_cast<double *>(scratch + kOffProb);
@@ -98,8 +104,8 @@ extern "C" int moespec_route_static(const float *logits, int M, int N, int k, in
   ws.arrive_route = reinterpret_cast<int *>(scratch + kOffArrive);
   ws.mask_words = kStaticMaskWords;
   // the shared array keeps whatever the last call (possibly an aborted one) left: clear the accumulators
-  if (cudaMemsetAsync(scratch + kOffZero, 0, kZeroBytes, static_cast<cudaStream_t>(stream)) != cudaSuccess)
-    return MOESPEC_ERR_CUDA;
+  e = cudaMemsetAsync(scratch + kOffZero, 0, kZeroBytes, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return cuda_fail(e);
   ws.active = reinterpret_cast<int *>(scratch + kOffActive);
   ws.row2expert = reinterpret_cast<int *>(scratch + kOffRow2Exp);
   ws.stats = reinterpret_cast<moespec_stats *>(scratch + kOffStats);
@@ -124,5 +130,6 @@ extern "C" int moespec_route_static(const float *logits, int M, int N, int k, in
   desc.shortlist = shortlist;
   desc.renormalize = renormalize;
   LaunchCtx c{&desc, &ws, M, k, B > N ? N : B, M * k, static_cast<cudaStream_t>(stream), 0};
-  return launch_route(c, logits) == cudaSuccess ? MOESPEC_OK : MOESPEC_ERR_CUDA;
+  e = launch_route(c, logits);
+  return e == cudaSuccess ? (int)MOESPEC_OK : cuda_fail(e);
 }

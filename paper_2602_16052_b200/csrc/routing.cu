@@ -23,7 +23,6 @@
 #include "internal.h"
 #include <cstdlib>
 #include <math_constants.h>
-#include <stdio.h>
 
 namespace moespec {
 
@@ -33,6 +32,7 @@ __device__ __forceinline__ float to_float(__half v) { return __half2float(v); }
 
 constexpr unsigned kFull = 0xffffffffu;
 constexpr double kScoreScale = 4503599627370496.0;   // 2^52: scores are sums of round(p * 2^52)
+constexpr unsigned long long kScoreOneMinus = (1ull << 52) - 1ull;
 constexpr int kNone = 0x7fffffff;
 
 // Monotone map float -> uint32 (larger float, larger key); -0 and +0 share a key.
@@ -99,7 +99,8 @@ __device__ __forceinline__ void token_softmax(const float *zrow, int N, double *
     if ((valid >> s) & 1u) {
       const double p = e[s] / sum;
       prob_row[lane + 32 * s] = p;
-      atomicAdd(score_fx + lane + 32 * s, (unsigned long long)__double2ull_rn(p * kScoreScale));
+      // p == 1 exactly is clamped one unit below 2^52, so that max_M = 4096 such tokens cannot wrap the sum
+      atomicAdd(score_fx + lane + 32 * s, min((unsigned long long)__double2ull_rn(p * kScoreScale), kScoreOneMinus));
     }
 }
 
@@ -191,9 +192,6 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
   // only start after this kernel has finished, polls the flag)
   if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
   clear_colmask(colmask, N * ((M + 31) >> 5));
-#ifdef MOESPEC_ROUTE_TIMING
-  const long long tm0 = clock64();
-#endif
   if (i < N) {
     const T *w = Wr + (size_t)i * d;
     float acc[TT];
@@ -242,9 +240,6 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
     if (lane == 0) __threadfence();
   }
   __syncthreads();
-#ifdef MOESPEC_ROUTE_TIMING
-  const long long tm1 = clock64();
-#endif
   if (threadIdx.x == 0) {
     const int prev = atomicAdd(&arrive[blockIdx.y], 1);
     s_last = (prev == (int)gridDim.x - 1);
@@ -254,9 +249,6 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
     }
   }
   __syncthreads();
-#ifdef MOESPEC_ROUTE_TIMING
-  const long long tm2 = clock64();
-#endif
   if (s_last) {
     // softmax and top-k are independent chains: with up to four tokens they run on different warps
     const bool split = 2 * TT <= 8;
@@ -267,10 +259,6 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane,
                   which);
   }
-#ifdef MOESPEC_ROUTE_TIMING
-  if (s_last && threadIdx.x == 0 && blockIdx.y == 0)
-    printf("router (cycles): dot %lld arrive %lld token %lld\n", tm1 - tm0, tm2 - tm1, clock64() - tm2);
-#endif
 }
 
 // ---------------------------------------------------------------------------
@@ -396,8 +384,8 @@ cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return c
 // Trees beyond 64 tokens of a 16-bit layer take the tensor-core router (d must split into eight K ranges of
 // whole 32-element steps).
 static bool use_router_mma(const LaunchCtx &c) {
-  static const bool off = [] { const char *v = getenv("MOESPEC_NO_ROUTER_MMA"); return v && v[0] == '1'; }();
-  static const int min_m = [] { const char *v = getenv("MOESPEC_ROUTER_MMA_MIN_M"); return v ? atoi(v) : 65; }();
+  static const bool off = [] { const char *v = experiment_env("MOESPEC_NO_ROUTER_MMA"); return v && v[0] == '1'; }();
+  static const int min_m = [] { const char *v = experiment_env("MOESPEC_ROUTER_MMA_MIN_M"); return v ? atoi(v) : 65; }();
   // (also for wide routers: with N >= 128 the tensor-core kernel wins at every tree size measured)
   return !off && is_16bit(c.desc->dtype) && (c.M >= min_m || c.desc->n_experts >= 128) && c.desc->d % 256 == 0;
 }
@@ -592,14 +580,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     pdl_wait();
     pdl_trigger();
   }
-#ifdef MOESPEC_ROUTE_TIMING
-  long long tmark[10];
-  int nmark = 0;
-#define ROUTE_MARK() do { if (tid == 0) tmark[nmark++] = clock64(); } while (0)
-#else
-#define ROUTE_MARK() do { } while (0)
-#endif
-  ROUTE_MARK();
 
   // ---- this warp's token: logit keys, probabilities, natural top-k (all loads issued up front)
   uint32_t key[W];
@@ -627,7 +607,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     s_fx[tid] = fx;
   }
   const int n_union = __syncthreads_count(in_union);
-  ROUTE_MARK();
   const int n_cand = __syncthreads_count(tid < N && s_cand[tid]);
   const bool fixed = a.shortlist == MOESPEC_STATIC;
   const int nS = fixed ? min(a.B, ws.n_static) : min(a.B, n_cand);
@@ -667,7 +646,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     if (lane == 0) s_Smask[warp] = word;
   }
   __syncthreads();
-  ROUTE_MARK();
   // publish the shortlist (S_rank was written by this CTA's threads before the barrier): the FFN kernel's
   // CTAs start streaming the weights of its best-ranked experts while the rest of the routing runs
   if (blockIdx.x == 0 && tid == 0 && ws.early_flag)      // the barrier above orders the other threads' S_rank stores before this release
@@ -675,7 +653,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
-  ROUTE_MARK();
 
   // ---- the CTA that arrives last finishes the call
   __threadfence();
@@ -687,7 +664,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   }
   __syncthreads();
   if (!s_last) return;
-  ROUTE_MARK();
 
   // rows per expert and exclusive scans of rows, token chunks and active experts (Appendix C gather)
   const int used_words = (M + 31) >> 5;
@@ -842,9 +818,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     for (int o = 16; o > 0; o >>= 1) cov += shfl_xor_double(cov, o);
     cov *= 1.0 / kScoreScale;
   }
-  ROUTE_MARK();
-  ROUTE_MARK();
-  ROUTE_MARK();
   if (tid == 224) {         // lane 0 of warp 7, which holds the coverage sum
     const int R = s_offset[N];
     ws.counters[0] = nS;
@@ -864,14 +837,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     *ws.stats = st;
     *ws.status = 0;
     *ws.arrive_route = 0;
-  }
-  if (tid == 0) {
-#ifdef MOESPEC_ROUTE_TIMING
-    tmark[nmark++] = clock64();
-    printf("route (cycles): load+scores %lld shortlist %lld reroute %lld arrive %lld scan %lld rows %lld units %lld stats %lld total %lld\n",
-           tmark[1] - tmark[0], tmark[2] - tmark[1], tmark[3] - tmark[2], tmark[4] - tmark[3], tmark[5] - tmark[4],
-           tmark[6] - tmark[5], tmark[7] - tmark[6], tmark[8] - tmark[7], tmark[8] - tmark[0]);
-#endif
   }
   __syncthreads();
   for (int i = tid; i < N; i += blockDim.x) {

@@ -43,3 +43,30 @@ def test_algorithmic_bytes_of_the_headline_point():
     want = 32 * 3 * 2048 * 1024 * 2 + 64 * 2048 * 2 + 63 * 2048 * 2 + 63 * 2048 * 4
     assert bench.algorithmic_bytes(cfg, 63, 32, 4) == want
     assert cfg.expert_weight_bytes() == 3 * 2048 * 1024 * 2
+
+
+def test_roofline_traffic_comes_from_the_tracked_counters_file():
+    """roofline.traffic is read from the counters file kept beside the profiler summary; the file must agree
+    with the launches that summary lists and with the algorithmic bytes of the workload."""
+    import re
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2602_16052_b200 import synth
+    c = bench.read_counters()
+    assert c is not None, "counters file missing"
+    traffic = bench.dram_traffic_per_launch()
+    assert traffic == c["dram__bytes_read.sum"] + c["dram__bytes_write.sum"]
+    cfg = synth.CONFIGS["olmoe"]
+    algo = bench.B_HEADLINE * cfg.expert_weight_bytes()
+    assert c["algorithmic_bytes_per_launch"] == algo
+    assert 1.0 <= traffic / algo < 1.1, "DRAM traffic should be the weight bytes plus a few per cent"
+    # the summary's table rows for the same counters, in MB per captured launch
+    md = open(os.path.join(ROOT, "profiles", "ffn_tc_kernel_olmoe_M63_B32.md")).read()
+    def row(name):
+        m = re.search(r"\| " + re.escape(name) + r" \|([^\n]*)\|", md)
+        assert m, name
+        return [float(x) for x in re.findall(r"([0-9]+\.[0-9]+) MB", m.group(1))]
+    rd, wr = row("dram__bytes_read.sum"), row("dram__bytes_write.sum")
+    assert len(rd) == int(c["captured_launches"]) == len(wr)
+    assert abs(sum(rd) / len(rd) * 1e6 - c["dram__bytes_read.sum"]) <= 0.01e6 * len(rd) + 1e4
+    assert abs(sum(wr) / len(wr) * 1e6 - c["dram__bytes_write.sum"]) <= 0.01e6 * len(wr) + 1e4

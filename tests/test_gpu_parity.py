@@ -32,16 +32,24 @@ def make_layer(case, max_M, max_k, **kw):
                       max_M=max_M, max_k=max_k, **kw)
 
 
-def check_out(out, ref, dtype):
+def check_out(out, ref, dtype, scale_rows="all"):
+    """max |err| against tol * RMS(reference output).  The RMS is taken over ALL rows of the reference, the
+    scale the bar is stated on; rows the truncation policy zeroed (Section 3.3) must be exact zeros.  The ratio
+    against the RMS of the rows that do have an output is printed beside it as a diagnostic.  scale_rows="live"
+    is for the one constructed fixture in which most rows are zeroed (see that test)."""
     o = out.to("cpu", torch.float64).numpy()
-    # RMS over the tokens that received an expert: rows the policy zeroed (Section 3.3) must be exact zeros and
-    # would otherwise deflate the scale the tolerance is stated against
     live = np.any(ref != 0.0, axis=1)
     assert not np.any(o[~live]), "a token with no kept expert must get exact zeros"
-    rms = float(np.sqrt(np.mean(ref[live] ** 2))) if live.any() else 0.0
+    rms_all = float(np.sqrt(np.mean(ref ** 2))) if ref.size else 0.0
+    rms_live = float(np.sqrt(np.mean(ref[live] ** 2))) if live.any() else 0.0
+    rms = rms_all if scale_rows == "all" else rms_live
+    err_max = float(np.max(np.abs(o - ref))) if ref.size else 0.0
+    if rms_all > 0:
+        print(f"max|err|/RMS: {err_max / rms_all:.4f} over all rows, {err_max / rms_live:.4f} over the "
+              f"{int(live.sum())}/{len(live)} rows with an output")
     if dtype in ("bf16", "fp16") and out.dtype == torch.float32:
         tol = BF16_TOL if dtype == "bf16" else FP16_TOL
-        err = float(np.max(np.abs(o - ref)))
+        err = err_max
         assert err <= tol * rms, f"max err {err:.3e} > {tol} * rms {rms:.3e}"
     elif dtype in ("bf16", "fp16"):
         # out stored in 16 bits: the bar plus the final rounding of the result itself
@@ -54,8 +62,26 @@ def check_out(out, ref, dtype):
         assert not bad.any(), f"{bad.sum()} elements beyond 1e-5 relative; worst {np.max(np.abs(o - ref) / bound):.2f}x"
 
 
+def near_tie_explains(r_own, r, z_ref, eb, k, cand):
+    """Is every difference between the oracle's selection on its own logits (r_own) and on the GPU's logits (r)
+    explained by a gap that the logit error eb = max |z_gpu - z_ref| can close?  Two logits within eb of their
+    reference can change order only if they are less than 2 eb apart.  A probability moves by at most eb / 2
+    when every logit moves by at most eb (|dp_i| <= 2 p_i (1 - p_i) eb), a score by at most M eb / 2, so two
+    scores can change order only if they are less than M eb apart (plus the fp64 rounding of the sums)."""
+    M = z_ref.shape[0]
+    if r_own["S"] != r["S"]:
+        _, sgap = H.selection_margins(r_own, k, cand)
+        return sgap < M * eb + 1e-12
+    zs = np.sort(z_ref.astype(np.float64), axis=1)
+    for t in range(M):
+        if r_own["assign"][t] != r["assign"][t] or r_own["topk"][t] != r["topk"][t]:
+            if float(np.min(np.diff(zs[t]))) >= 2 * eb:      # no pair of this token's logits is close enough
+                return False
+    return True
+
+
 def run_e2e(cfg, M, B, policy, mode, renorm, ffn_kernel, seed=0, k=None, case=None, layer=None, residual=False,
-            out_dtype=torch.float32):
+            out_dtype=torch.float32, scale_rows="all"):
     """Run the GPU layer, then the oracle on the GPU's own fp32 logits; also check the logits."""
     k = cfg.k if k is None else k
     case = case or H.make_case(cfg, M, seed)
@@ -69,11 +95,12 @@ def run_e2e(cfg, M, B, policy, mode, renorm, ffn_kernel, seed=0, k=None, case=No
     z_gpu = layer.get_logits()
     z_ref = orc.router_logits(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]))
     zerr = 3e-6 if cfg.dtype == "fp32" else 2e-5
-    assert np.max(np.abs(z_gpu.astype(np.float64) - z_ref)) <= zerr * max(1.0, np.abs(z_ref).max())
+    eb = float(np.max(np.abs(z_gpu.astype(np.float64) - z_ref)))      # the logit error of this run
+    assert eb <= zerr * max(1.0, np.abs(z_ref).max())
     r = H.oracle_run(case, k, B, policy, mode, renorm, logits=z_gpu)
     H.compare_routing(layer.get_routing(), r, policy, k)
     ref = r["out"] + (H.f64(case["hidden"]) if residual else 0.0)
-    check_out(out, ref, cfg.dtype)
+    check_out(out, ref, cfg.dtype, scale_rows)
     assert st["n_union"] == len(r["union"]) and st["n_shortlist"] == len(r["S"])
     assert st["n_active"] == len(r["active"]) and st["n_rows"] == len(r["perm_row2tok"])
     assert st["n_dropped"] == M * k - st["n_rows"]
@@ -82,8 +109,9 @@ def run_e2e(cfg, M, B, policy, mode, renorm, ffn_kernel, seed=0, k=None, case=No
     # the oracle on its own logits makes the same selection unless a near-tie sits inside the logit error
     r_own = H.oracle_route(z_ref, k, B, policy, mode, renorm)
     if r_own["S"] != r["S"] or r_own["assign"] != r["assign"]:
-        zgap, sgap = H.selection_margins(r_own, min(k, cfg.n_experts), None if mode == orc.FROM_ALL else r_own["union"])
-        assert min(zgap, sgap) < 1e-4, "selection differs from the oracle's without a certified near-tie"
+        cand = None if mode == orc.FROM_ALL else r_own["union"]
+        assert near_tie_explains(r_own, r, z_ref, eb, min(k, cfg.n_experts), cand), \
+            "selection differs from the oracle's and no gap below the measured logit error explains it"
     if own:
         layer.destroy()
     return out, r, st
@@ -245,9 +273,20 @@ def test_seeded_sweep_of_random_shapes_and_settings():
 
 
 def test_qwen3_shape_layer():
+    """Single layers at the full Qwen3-30B-A3B shape (Table 3), raw gating as that architecture uses and
+    renormalised as the benchmark tables run it."""
     cfg = synth.CONFIGS["qwen3"]
-    for M, B in ((63, 32), (127, 128)):
-        run_e2e(cfg, M, B, orc.SUBSTITUTION, orc.FROM_ALL, False, ms().FFN_TENSOR_CORE)
+    for M, B, renorm in ((63, 32, False), (127, 128, False), (63, 64, True), (63, 32, True)):
+        run_e2e(cfg, M, B, orc.SUBSTITUTION, orc.FROM_ALL, renorm, ms().FFN_TENSOR_CORE)
+
+
+def test_olmoe_largest_tree_full_width():
+    """The largest tree of the stack sweep at the full OLMoE shape: M = 511, f = 1024, B = 32 and unbudgeted."""
+    cfg = synth.CONFIGS["olmoe"]
+    case = H.make_case(cfg, 511, seed=511)
+    for B in (32, 64):
+        out, r, st = run_e2e(cfg, 511, B, orc.SUBSTITUTION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, case=case)
+        assert st["n_rows"] == 511 * cfg.k
 
 
 def test_mixtral_shape_layer_reduced_width():
@@ -259,7 +298,12 @@ def test_mixtral_shape_layer_reduced_width():
 
 def test_truncation_zero_rows_and_budget_below_k():
     cfg = synth.CONFIGS["olmoe"].with_(f=128, slope=0.0)      # flat routing: no expert is in every top-k
-    out, r, st = run_e2e(cfg, 63, 1, orc.TRUNCATION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE)
+    # With one kept expert and flat routing the policy zeroes about seven rows of eight.  Zero rows are exact on
+    # both sides and carry no error, but they shrink the all-rows RMS by sqrt(live fraction) ~ 0.35, so the
+    # rounding error of the rows that do have an output (~1e-2 of THEIR RMS, the same as in every other test)
+    # would be measured against a scale that the zeroing, not the arithmetic, set.  This fixture alone states
+    # its bound on the rows with an output; both ratios are printed.
+    out, r, st = run_e2e(cfg, 63, 1, orc.TRUNCATION, orc.FROM_ALL, True, ms().FFN_TENSOR_CORE, scale_rows="live")
     empty = [t for t in range(63) if not r["assign"][t]]
     assert empty, "fixture should drop every expert of some token"
     assert not out[empty].float().abs().max().item() > 0      # exact zeros
@@ -425,20 +469,23 @@ def test_bounded_wait_expires_cleanly_and_layer_recovers():
 
 
 # ------------------------------------------------------------------ full Mixtral-shaped layer, sampled tokens
-def test_mixtral_full_shape_sampled_tokens():
+@pytest.mark.parametrize("M,B,ffn", [(15, 4, "tensor_core"), (63, 6, "tensor_core"), (63, 8, "tensor_core"),
+                                     (15, 4, "cuda_core")])
+def test_mixtral_full_shape_sampled_tokens(M, B, ffn):
     """d=4096, f=14336, N=8, k=2 at full size.  Routing is checked for every token; layer outputs are
-    checked for sampled tokens, whose experts the oracle evaluates one at a time."""
+    checked for sampled tokens, whose experts the oracle evaluates one at a time.  The CUDA-core case stages
+    rows of f floats (57 KB) in shared memory, beyond the default limit of a kernel."""
     m = ms()
     cfg = synth.CONFIGS["mixtral"]
-    M, B = 15, 4
     case = H.make_case(cfg, M, seed=5)
-    layer = make_layer(case, M, cfg.k, out_dtype=torch.float32)
+    layer = make_layer(case, M, cfg.k, out_dtype=torch.float32,
+                       ffn_kernel=m.FFN_TENSOR_CORE if ffn == "tensor_core" else m.FFN_CUDA_CORE)
     out = layer.verify_layer(case["hidden"], cfg.k, B)
     torch.cuda.synchronize()
     assert layer.get_stats()["status"] == 0
     r = H.oracle_route(layer.get_logits(), cfg.k, B, orc.SUBSTITUTION, orc.FROM_ALL, True)
     H.compare_routing(layer.get_routing(), r, orc.SUBSTITUTION, cfg.k)
-    sample = [0, 7, 14]
+    sample = [0, M // 2, M - 1]
     Hs = H.f64(case["hidden"][sample])
     ref = np.zeros((len(sample), cfg.d))
     for e in sorted({i for t in sample for i in r["assign"][t]}):
@@ -540,3 +587,27 @@ def test_fp16_layer(ffn):
     run_e2e(cfg, 63, 32, orc.SUBSTITUTION, orc.FROM_ALL, True, kern, case=case)
     run_e2e(cfg, 63, 12, orc.TRUNCATION, orc.FROM_UNION, False, kern, case=case, out_dtype=torch.float16,
             residual=True)
+
+
+# ------------------------------------------------------------------ limits of the score representation
+def test_scores_do_not_wrap_when_one_expert_takes_every_token():
+    """Scores (Eq. 5) are sums of round(p * 2^52) in 64 bits.  With max_M = 4096 tokens that all give one expert
+    p == 1.0 in fp64 the plain sum would reach 2^64 and wrap to zero, and the dominant expert would rank last.
+    (Every other expert then has p < 2^-53 per token, below the resolution of the representation: their order
+    among themselves is the tie order, so only what is unique is compared for B > 1.)"""
+    cfg = synth.LayerConfig("wrap", d=128, n_experts=8, k=2, f=128, dtype="bf16", slope=0.0)
+    M = 4096
+    case = H.make_case(cfg, 4, seed=1)
+    z = np.zeros((M, cfg.n_experts), dtype=np.float32)
+    z[:, 5] = 60.0                       # exp(-60) vanishes against 1: p_5 == 1.0 exactly
+    z[:, 2] = 1.0
+    layer = make_layer(case, max_M=M, max_k=2, ffn_kernel=ms().FFN_CUDA_CORE)
+    r = H.oracle_route(z, 2, 1, orc.SUBSTITUTION, orc.FROM_ALL, True)
+    assert r["S"] == [5] and r["score"][5] == float(M)
+    layer.route_from_logits(torch.from_numpy(z).cuda(), 2, 1)
+    H.compare_routing(layer.get_routing(), r, orc.SUBSTITUTION, 2)
+    layer.route_from_logits(torch.from_numpy(z).cuda(), 2, 8)
+    g = layer.get_routing()
+    assert g["S"][0] == 5 and sorted(g["S"]) == list(range(8))
+    assert np.all(g["assign_idx"] == np.array([5, 2])) and abs(g["score"][5] - M) <= M * 2.0 ** -52
+    layer.destroy()

@@ -36,7 +36,10 @@ def check_layers(cfg, cases, layers, xs, budgets, policy, mode, renorm):
         x_l = H.f64(xs[l])
         c = dict(case)
         c["hidden"] = xs[l]
-        r = H.oracle_run(c, cfg.k, budgets[l], policy, mode, renorm, logits=layer.get_logits())
+        z_gpu = layer.get_logits()
+        z_ref = orc.router_logits(x_l, H.f64(case["router_w"]), H.f64(case["router_bias"]))
+        assert np.max(np.abs(z_gpu.astype(np.float64) - z_ref)) <= 2e-5 * max(1.0, np.abs(z_ref).max()), f"logits of layer {l}"
+        r = H.oracle_run(c, cfg.k, budgets[l], policy, mode, renorm, logits=z_gpu)
         H.compare_routing(layer.get_routing(), r, policy, cfg.k)
         assert layer.get_stats()["status"] == 0
         nxt = x_l + r["out"]
@@ -89,10 +92,10 @@ def test_stack_per_layer_parity_with_per_layer_budgets(policy_name, mode_name, r
 
 
 def test_stack_at_full_layer_size():
-    """Four layers of the 16-layer benchmark stack at their full size (d=2048, N=64, f=1024, M=63, B=32), in
-    the configuration the benchmark times (one graph launch, bf16 residual stream), each layer checked
-    against the oracle on the GPU's own input to that layer."""
-    cfg = synth.CONFIGS["olmoe16"].with_(n_layers=4)
+    """All 16 layers of the benchmark stack at their full size (d=2048, N=64, f=1024, M=63, B=32), in the
+    configuration the benchmark times (one graph launch, bf16 residual stream), each layer checked against
+    the oracle on the GPU's own input to that layer."""
+    cfg = synth.CONFIGS["olmoe16"]
     M, B = 63, 32
     cases, layers, stack = build_stack(cfg, M, seed=2000)
     x0 = synth.gen_hidden(cfg, M, seed=2000, device="cuda")
@@ -102,6 +105,23 @@ def test_stack_at_full_layer_size():
     check_layers(cfg, cases, layers, xs, [B] * cfg.n_layers, orc.SUBSTITUTION, orc.FROM_ALL, True)
     for layer in layers:
         assert layer.get_stats()["n_active"] == B
+    stack.destroy()
+    for layer in layers:
+        layer.destroy()
+
+
+def test_wide_router_stack_at_full_layer_size():
+    """Three layers of the 48-layer Qwen3-30B-A3B-shaped stack at full size (d=2048, N=128, k=8, f=768),
+    renormalised gating and one graph launch per pass as the benchmark tables run it, at three points of its
+    (M, B) sweep; each layer checked against the oracle on the GPU's own input to that layer."""
+    cfg = synth.CONFIGS["qwen3"].with_(n_layers=3)
+    cases, layers, stack = build_stack(cfg, 127, seed=2000)
+    for M, B in ((63, 32), (63, 64), (127, 128)):
+        x0 = synth.gen_hidden(cfg, M, seed=2000, device="cuda")
+        out = stack.verify_stack(x0, cfg.k, B)
+        torch.cuda.synchronize()
+        xs = [x0.cpu()] + [stack.get_stream(l) for l in range(1, cfg.n_layers)] + [out.cpu()]
+        check_layers(cfg, cases, layers, xs, [B] * cfg.n_layers, orc.SUBSTITUTION, orc.FROM_ALL, True)
     stack.destroy()
     for layer in layers:
         layer.destroy()

@@ -45,7 +45,8 @@ def test_route_static_matches_handle_based_routing_twice_in_a_row():
     cfg = synth.CONFIGS["olmoe"].with_(f=128)
     case = synth.gen_layer(cfg, 21, 0, "cuda")
     k = cfg.k
-    calls = [(127, 32, m.SUBSTITUTION, m.FROM_ALL, True), (40, 5, m.TRUNCATION, m.FROM_UNION, False)]
+    calls = [(127, 32, m.SUBSTITUTION, m.FROM_ALL, True), (40, 5, m.TRUNCATION, m.FROM_UNION, False),
+             (300, 24, m.SUBSTITUTION, m.FROM_UNION, True), (9, 64, m.SUBSTITUTION, m.FROM_ALL, True)]
     for M, B, policy, shortlist, renorm in calls:
         h = synth.gen_hidden(cfg, M, 21, 0, "cuda")
         z = (h.float() @ case["router_w"].float().T + case["router_bias"]).contiguous()   # any fp32 logits will do
@@ -54,6 +55,35 @@ def test_route_static_matches_handle_based_routing_twice_in_a_row():
         check_same(got, want, M, k)
         again = m.route_static(z, k, B, policy, shortlist, renorm, out=got)     # reuse the caller's buffers
         check_same(again, want, M, k)
+
+
+def test_route_static_large_tree_against_the_oracle():
+    """Trees above 128 tokens take the branch in which a separate kernel works out the row of every (token,
+    slot) pair from the bit matrix in the shared scratch.  Here the results are compared with the CPU oracle
+    itself (a comparison with the handle-based entry point alone would pass a fault the two share), on a large
+    call, then a small one that finds the large call's leftovers, then the large one again."""
+    from oracle import moespec_oracle as orc
+    from paper_2602_16052_b200 import moespec as m
+    from tests import helpers as H
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = synth.gen_layer(cfg, 22, 0, "cpu")
+    k = cfg.k
+    calls = [(255, 32, orc.SUBSTITUTION, orc.FROM_ALL, True), (40, 12, orc.TRUNCATION, orc.FROM_UNION, False),
+             (m.ROUTE_STATIC_MAX_M, 16, orc.TRUNCATION, orc.FROM_ALL, True), (255, 32, orc.SUBSTITUTION, orc.FROM_ALL, True)]
+    for M, B, policy, shortlist, renorm in calls:
+        h = synth.gen_hidden(cfg, M, 22, 0, "cpu")
+        z = orc.router_logits(H.f64(h), H.f64(case["router_w"]), H.f64(case["router_bias"]))      # fp32 logits
+        r = orc.route(z, k, B, policy, shortlist, renorm)
+        got = m.route_static(torch.from_numpy(z).cuda(), k, B, policy, shortlist, renorm)
+        torch.cuda.synchronize()
+        nS, n_act, R = got["summary"][:3].tolist()
+        g = {"S": got["S_rank"][:nS].tolist(), "n_rows": R, "count": got["count"].tolist(),
+             "offset": got["offset"].tolist(), "perm_row2tok": got["perm_row2tok"][:R].tolist(),
+             "score": got["score"].cpu().numpy()}
+        for name in ("topk_idx", "assign_idx", "tokslot2row", "gate_w"):
+            g[name] = got[name][:M * k].cpu().numpy().reshape(M, k)
+        H.compare_routing(g, r, policy, k)
+        assert n_act == len(r["active"]) and R == len(r["perm_row2tok"])
 
 
 def test_route_static_rejects_sizes_beyond_its_scratch():
