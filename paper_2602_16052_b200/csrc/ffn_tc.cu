@@ -15,22 +15,28 @@
 //   down unit:     D = W2[e, slab, :] H_e^T,     y[row, slab] = D  (fp32)
 //
 // One launch covers both kinds.  The unit list holds every gate/up unit, then
-// every down unit; persistent CTAs (one per SM) draw units in list order from a
-// global dispenser, so the gate/up tail overlaps the start of the down
-// projection.  A down unit needs all of its expert chunk's h_mid: each finished
-// gate/up unit bumps a per-chunk ready counter (release), and the producer of a
-// down unit waits (bounded, acquire) for the counter to reach the slab count.
-// Units are handed out in order and gate/up units never wait, so every unit a
-// down unit waits for is already running or done: there is no circular wait.
+// every down unit; persistent CTAs (one per SM) draw EVERY unit, the first one
+// included, as a ticket from a global dispenser, in list order, so the gate/up
+// tail overlaps the start of the down projection.  A down unit needs all of its
+// expert chunk's h_mid: each finished gate/up unit bumps a per-chunk ready
+// counter (release), and the producer of a down unit waits (bounded, acquire)
+// for the counter to reach the slab count.  Tickets are handed out in order to
+// CTAs that are running, and gate/up units never wait, so every unit a down
+// unit waits for has been drawn by a running CTA or is done: there is no
+// circular wait, however the grid is placed on the SMs (a CTA that becomes
+// resident late simply draws a later ticket, e.g. when another handle's kernel
+// holds some of the SMs).  The dispenser and the down-unit counter are zeroed
+// by the router kernel of the call, which completes before this kernel starts.
 //
 // Early start (trees of up to 128 tokens): the CTAs of this kernel are resident
-// while the routing kernels still run.  CTA c does not wait for them: as soon as
-// the routing kernel has published the shortlist (a flag; at once when the
-// shortlist is fixed) it starts on gate/up unit c of the rank-ordered list --
-// expert S_rank[c / slabs], slab c % slabs -- with ALL tokens of the tree as the
-// B operand, read from `hidden` itself, and keeps the routed tokens' columns in
-// the epilogue, by which time the gather order exists.  The routing kernel lists
-// the units in the same order, so unit c of the list is that unit.
+// while the routing kernels still run.  A CTA whose first ticket c is below the
+// grid size does not wait for them: as soon as the routing kernel has published
+// the shortlist (a flag; at once when the shortlist is fixed) it starts on
+// gate/up unit c of the rank-ordered list -- expert S_rank[c / slabs], slab
+// c % slabs -- with ALL tokens of the tree as the B operand, read from `hidden`
+// itself, and keeps the routed tokens' columns in the epilogue, by which time
+// the gather order exists.  The routing kernel lists the units in the same
+// order, so unit c of the list is that unit.
 //
 // Ten warps per CTA:
 //   warp 0        : dispenser + TMA producer.  Lane 0 waits and draws units; all
@@ -102,7 +108,7 @@ struct TcArgs {
   int M, k, residual, out_is_fp32;
   long long spin_limit; // cycles after which any wait gives up
   // early start (see the kernel's header comment)
-  int early;                 // 1: CTA c begins with gate/up unit c of the shortlist before routing has finished
+  int early;                 // 1: tickets below the grid size are started on before routing has finished
   const int *early_flag;     // 0 until the routing kernel has published the shortlist, then |S| + 1
   const int *S_rank;         // shortlist in rank order
   const int *perm_row2tok;   // gather order: row -> token
@@ -302,7 +308,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     // ===================================================== dispenser + TMA producer
     // Lane 0 owns every wait and the queue; the copies of a stage are issued by all lanes (one box
     // each), because a single thread issuing 8-16 copies per stage would cap the SM's streaming rate.
-    // CTA b starts with unit b; later units come from the dispenser.  The next unit is drawn a few
+    // Every unit, the first included, is a ticket from the dispenser.  The next unit is drawn a few
     // stages before the current one ends: early enough that the atomic and the descriptor load are
     // hidden behind the stages still in flight, late enough that no CTA sits on units others could run.
     int n_total = 0;                 // valid once `waited`
@@ -314,12 +320,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     sentinel.expert = -1; sentinel.tile = 0; sentinel.row0 = 0; sentinel.n_rows = 0; sentinel.chunk = 0;
     sentinel.phase = 0; sentinel.pad0 = 0; sentinel.pad1 = 0;
     Unit un = sentinel;
+    // the first ticket (the router kernel of this call left the dispenser at zero)
+    int t_first = 0;
+    if (lane == 0) t_first = atomicAdd(a.unit_counter, 1);
     if (a.early) {
-      // The routing kernel publishes the shortlist long before the gather order exists.  CTA c starts on
-      // gate/up unit c of the rank-ordered list (expert S_rank[c / tiles], slab c % tiles) with ALL tokens
-      // as the MMA's N dimension, read straight from `hidden`; the epilogue keeps the routed tokens only.
-      // The routing kernel builds the unit list in the same order, so unit c of the list is this unit.
-      if (lane == 0) {
+      // The routing kernel publishes the shortlist long before the gather order exists.  Ticket c below the
+      // grid size is gate/up unit c of the rank-ordered list (expert S_rank[c / tiles], slab c % tiles) and
+      // is started on with ALL tokens as the MMA's N dimension, read straight from `hidden`; the epilogue
+      // keeps the routed tokens only.  The routing kernel builds the unit list in the same order and keeps
+      // the experts of those ranks in it even without rows, so unit c of the list is this unit.
+      if (lane == 0 && t_first < (int)gridDim.x) {
         int fl = a.static_nS + 1;        // a fixed shortlist needs no publication: stream from the first cycle
         const int *rank = a.static_nS > 0 ? a.static_order : a.S_rank;
         if (a.static_nS == 0) {
@@ -329,22 +339,23 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
             __nanosleep(32);
           }
         }
-        if (ok && (int)blockIdx.x < (fl - 1) * a.tiles_real) {
-          un.expert = __ldcg(rank + blockIdx.x / a.tiles_real);
-          un.tile = blockIdx.x % a.tiles_real;
+        if (ok && t_first < (fl - 1) * a.tiles_real) {
+          un.expert = __ldcg(rank + t_first / a.tiles_real);
+          un.tile = t_first % a.tiles_real;
           un.n_rows = a.M;
           un.pad0 = 1;                 // dense: every token, rows of `hidden`
+          un.pad1 = t_first;           // its place in the unit list
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (ok && !__shfl_sync(0xffffffffu, un.pad0, 0)) {      // no early unit for this CTA: wait like everybody
+      if (ok && !__shfl_sync(0xffffffffu, un.pad0, 0)) {      // no early unit for this ticket: wait like everybody
         pdl_wait();
         waited = true;
       }
     }
     if (waited) {
       n_total = a.n_units[0] + a.n_units[1];
-      if (lane == 0 && (int)blockIdx.x < n_total) un = a.units[blockIdx.x];
+      if (lane == 0 && !un.pad0 && t_first < n_total) un = a.units[t_first];
     }
     while (ok) {
       Unit un_next = sentinel;
@@ -354,7 +365,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         // to stream; a down unit still counts as done
         while (un.expert >= 0 && un.n_rows == 0 && !un.pad0) {
           if (un.phase == 1) atomicAdd(a.down_done, 1);
-          const int u2 = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
+          const int u2 = atomicAdd(a.unit_counter, 1);
           un = u2 < n_total ? a.units[u2] : sentinel;
         }
         const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
@@ -408,7 +419,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           n_total = a.n_units[0] + a.n_units[1];
         }
         if (lane == 0) {
-          if (kc == draw_at) u_next = (int)gridDim.x + atomicAdd(a.unit_counter, 1);
+          if (kc == draw_at) u_next = atomicAdd(a.unit_counter, 1);
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
           else mbar_expect_tx(full, tx);
         }
@@ -549,7 +560,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         // h_mid the expert owns and the gather order says which token each row is.
         pdl_wait();
         const int et = (int)threadIdx.x - 64;
-        Unit real = a.units[blockIdx.x];
+        Unit real = a.units[un.pad1];
         if (real.expert != un.expert || real.tile != un.tile || real.phase != 0 || real.n_rows > kMaxTokChunk) {
           if (et == 0) atomicExch(a.status, (int)MOESPEC_ERR_INTERNAL);      // the two kernels disagree on the list
           real.n_rows = 0;

@@ -76,7 +76,7 @@ struct Workspace {
   int *static_order;        // [N] the fixed ordering itself: expert at position r (first n_static entries)
   Unit *units;          // gate/up units (expert, chunk, tile ascending) followed by the down units
   int *ready;           // [chunks] gate/up units finished per (expert, token chunk); zeroed by the route kernel
-  int *unit_counter;    // [0] next unit to hand out, [1] finished down units; zeroed by the route kernel
+  int *unit_counter;    // [0] next unit to hand out, [1] finished down units; zeroed by the router kernel
   int *counters;        // [0]=n_S [1]=n_active [2]=R [3]=n_units_up [4]=n_units_down
   moespec_stats *stats; // device copy
   int *status;          // device status word (0 = ok)

@@ -155,6 +155,23 @@ __device__ __forceinline__ void clear_colmask(unsigned *colmask, int words) {
   for (int i = cta * blockDim.x + threadIdx.x; i < words; i += n_cta * blockDim.x) colmask[i] = 0u;
 }
 
+// The FFN kernel's control words must be in their initial state when its first CTA starts: the shortlist flag
+// at 0 (the routing kernel publishes the call's shortlist later; the FFN kernel polls the flag), its unit
+// dispenser and its down-unit counter at 0.  The router kernel's first CTA sets them: it runs after the
+// previous call's FFN kernel has completed (it has just waited for that) and completes before this call's FFN
+// kernel can start -- except with a fixed shortlist, where the FFN kernel is released right behind this kernel's
+// CTAs: there the stores are performed (fence) before this CTA releases the dependents.
+__device__ __forceinline__ void reset_ffn_control(int *early_flag, int *unit_counter, int fence_reset) {
+  if (!early_flag || blockIdx.x != 0 || blockIdx.y != 0) return;
+  if (threadIdx.x == 0) {
+    *early_flag = 0;
+    unit_counter[0] = 0;
+    unit_counter[1] = 0;
+    if (fence_reset) __threadfence();
+  }
+  if (fence_reset) __syncthreads();
+}
+
 // ---------------------------------------------------------------------------
 // K1: z[t,i] = b_i + w_i . h_t with fp32 accumulation, fused with the token's
 // softmax and top-k.  A CTA takes TT tokens x 8 experts; warp w owns expert w of
@@ -169,6 +186,7 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
                                                           const float *__restrict__ bias, float *logits,
                                                           double *prob, int *topk_idx, unsigned long long *score_fx,
                                                           int *natcnt, int *arrive, int *early_flag,
+                                                          int *unit_counter, int fence_reset,
                                                           unsigned *colmask, int M, int N, int d, int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t0 = blockIdx.y * TT;
@@ -185,12 +203,10 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       if ((lane + u * 32) * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(Wr + (size_t)i * d + (lane + u * 32) * VEC);
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  reset_ffn_control(early_flag, unit_counter, fence_reset);
   // Dependents are released only now: with a fixed shortlist the FFN kernel of this call starts at once,
   // and it reads `hidden`, which the previous kernel in the stream may have produced.
   pdl_trigger();
-  // the call's shortlist is not known yet (the routing kernel publishes it; the FFN kernel, which can
-  // only start after this kernel has finished, polls the flag)
-  if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
   clear_colmask(colmask, N * ((M + 31) >> 5));
   if (i < N) {
     const T *w = Wr + (size_t)i * d;
@@ -292,8 +308,9 @@ template <typename T>
 __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                          const float *__restrict__ bias, float *logits, double *prob,
                                                          int *topk_idx, unsigned long long *score_fx, int *natcnt,
-                                                         int *arrive, int *early_flag, unsigned *colmask, int M, int N,
-                                                         int d, int k) {
+                                                         int *arrive, int *early_flag, int *unit_counter,
+                                                         int fence_reset, unsigned *colmask, int M, int N, int d,
+                                                         int k) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, tg = lane & 3;
   const int e0 = blockIdx.x * kRmExperts, t0 = blockIdx.y * kRmTokens;
@@ -313,8 +330,8 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
     }
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
+  reset_ffn_control(early_flag, unit_counter, fence_reset);
   pdl_trigger();       // released only now: see router_topk_kernel
-  if (early_flag && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *early_flag = 0;
   clear_colmask(colmask, N * ((M + 31) >> 5));
   const T *hb = hidden + (size_t)min(t0 + g, M - 1) * d + warp * kw + tg * 8;
   float c[4] = {0.f, 0.f, 0.f, 0.f};
@@ -376,7 +393,8 @@ static cudaError_t launch_router_mma(const LaunchCtx &c, const void *hidden) {
   const dim3 grid((D.n_experts + kRmExperts - 1) / kRmExperts, (c.M + kRmTokens - 1) / kRmTokens);
   return launch_kernel(router_mma_kernel<T>, grid, dim3(256), 0, c.stream, (const T *)hidden, (const T *)D.router_w,
                        D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.score_fx, ws.natcnt_acc, ws.arrive,
-                       ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
+                       ws.early_flag, ws.unit_counter, D.shortlist == MOESPEC_STATIC ? 1 : 0, ws.colmask, c.M, D.n_experts,
+                       D.d, c.k);
 }
 template <>
 cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
@@ -406,14 +424,17 @@ static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
   if (c.M <= 64 && min_tt <= 2)
     return launch_kernel(router_topk_kernel<T, 2>, dim3(ex_tiles, (c.M + 1) / 2), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.unit_counter, D.shortlist == MOESPEC_STATIC ? 1 : 0,
+                         ws.colmask, c.M, D.n_experts, D.d, c.k);
   if (c.M <= 128 && min_tt <= 4)
     return launch_kernel(router_topk_kernel<T, 4>, dim3(ex_tiles, (c.M + 3) / 4), dim3(256), 0, c.stream,
                          (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
+                         ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.unit_counter, D.shortlist == MOESPEC_STATIC ? 1 : 0,
+                         ws.colmask, c.M, D.n_experts, D.d, c.k);
   return launch_kernel(router_topk_kernel<T, 8>, dim3(ex_tiles, (c.M + 7) / 8), dim3(256), 0, c.stream,
                        (const T *)hidden, (const T *)D.router_w, D.router_bias, ws.logits, ws.prob, ws.topk_idx,
-                       ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.colmask, c.M, D.n_experts, D.d, c.k);
+                       ws.score_fx, ws.natcnt_acc, ws.arrive, ws.early_flag, ws.unit_counter, D.shortlist == MOESPEC_STATIC ? 1 : 0,
+                         ws.colmask, c.M, D.n_experts, D.d, c.k);
 }
 
 cudaError_t launch_router_logits(const LaunchCtx &c, const void *hidden) {
@@ -781,10 +802,6 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       const int lt = tid - 128, nthr = 96;
       const int n_up = n_chunks * a.tiles_up, n_down = n_chunks * a.tiles_down;
       for (int i = lt; i < n_chunks; i += nthr) ws.ready[i] = 0;
-      if (lt == 0) {
-        ws.unit_counter[0] = 0;
-        ws.unit_counter[1] = 0;
-      }
       for (int u = lt; u < n_up + n_down; u += nthr) {
         const int phase = u >= n_up;
         const int tiles = phase ? a.tiles_down : a.tiles_up;

@@ -386,6 +386,29 @@ def test_device_entry_can_be_captured_into_a_callers_graph():
     layer.destroy()
 
 
+def test_two_handles_on_two_streams_at_once():
+    """Different handles are independent: their calls may overlap on the GPU.  The FFN kernels of the two
+    streams then share the SMs, so neither grid is resident as a whole; every work unit is a ticket drawn by
+    a running CTA, so both must finish with status 0 and the bits of a call that had the GPU to itself."""
+    cfg = synth.CONFIGS["olmoe"]
+    cases = [H.make_case(cfg, 63, seed=70 + i) for i in range(2)]
+    layers = [make_layer(c, 63, cfg.k, out_dtype=torch.float32) for c in cases]
+    alone = [L.verify_layer(c["hidden"], cfg.k, 32).clone() for L, c in zip(layers, cases)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    outs = [torch.empty_like(a) for a in alone]
+    for it in range(30):
+        for i in (0, 1):
+            layers[i].verify_layer(cases[i]["hidden"], cfg.k, 32 if it % 2 == 0 else 16, outs[i], streams[i])
+    for i in (0, 1):
+        layers[i].verify_layer(cases[i]["hidden"], cfg.k, 32, outs[i], streams[i])
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        assert layers[i].get_stats()["status"] == 0
+        assert torch.equal(outs[i], alone[i])
+        layers[i].destroy()
+
+
 # ------------------------------------------------------------------ argument errors (host side only)
 def test_argument_errors_return_codes():
     m = ms()
