@@ -15,6 +15,12 @@ Prints one JSON line.  With --gpus N > 1 (under torchrun) every rank runs an
 independent replica of the same workload on its own GPU (the layer has no
 data-path collective); time is the max over ranks.  --impl reference times the
 CPU oracle on the host cores instead.
+
+  --mode ep   (with --gpus N under torchrun) expert-parallel instead of replicas: rank r holds the weights of
+              its block of the experts only, every rank routes the same tree (replicated router, no exchange),
+              streams its resident kept experts and the partial outputs [M, d] fp32 are summed by one NCCL
+              all-reduce per layer, inside the timed region.  The job then processes K layers in total
+              ("scaling": "strong").
 """
 from __future__ import annotations
 
@@ -148,16 +154,98 @@ def algorithmic_bytes(cfg, M, n_active, out_bytes):
     return n_active * 3 * cfg.d * cfg.f * w + cfg.n_experts * cfg.d * w + M * cfg.d * w + M * cfg.d * out_bytes
 
 
-def build_layers(cfg, M, n_copies, device, out_dtype):
+def build_layers(cfg, M, n_copies, device, out_dtype, resident=None):
+    """resident = (first, count): only that block of every copy's experts is generated and held (expert-parallel)."""
     from paper_2602_16052_b200 import moespec
     layers, hiddens = [], []
+    experts = None if resident is None else range(resident[0], resident[0] + resident[1])
     for c in range(n_copies):
-        L = synth.gen_layer(cfg, seed=1000 + c, layer=0, device=device)
+        L = synth.gen_layer(cfg, seed=1000 + c, layer=0, device=device, experts=experts)
         hiddens.append(synth.gen_hidden(cfg, M, seed=1000 + c, layer=0, device=device))
         layers.append(moespec.Layer(L["router_w"], L["router_bias"], L["w_gate"], L["w_up"], L["w_down"], max_M=M,
                                     max_k=cfg.k, policy=moespec.SUBSTITUTION, shortlist=moespec.FROM_ALL,
-                                    renormalize=True, out_dtype=out_dtype))
+                                    renormalize=True, out_dtype=out_dtype, resident=resident))
     return layers, hiddens
+
+
+def run_expert_parallel(args, dist, device, rank, world, barrier):
+    """--mode ep: one layer split by experts over the ranks; per step every rank runs its shard and the partial
+    outputs are summed with one all-reduce.  Prints the benchmark line (rank 0)."""
+    from paper_2602_16052_b200 import ep
+    cfg = synth.CONFIGS[WORKLOAD]
+    M, k, B = M_TOKENS, cfg.k, B_HEADLINE
+    resident = ep.expert_range(rank, world, cfg.n_experts)
+    layers, hiddens = build_layers(cfg, M, args.copies, device, torch.float32, resident if world > 1 else None)
+    outs = [torch.empty((M, cfg.d), dtype=torch.float32, device=device) for _ in layers]
+    n = len(layers)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        layers[i % n].verify_layer(hiddens[i % n], k, B, outs[i % n], stream)
+        if world > 1:
+            dist.all_reduce(outs[i % n])          # sum of the shards' partial outputs, on every rank
+
+    sampler = ClockSampler(device.index or 0)
+    sampler.start()
+    time.sleep(0.3)
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+    torch.cuda.synchronize()
+    t0m = sampler.mark()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.stop(t0m, sampler.mark())
+    ms_total = job_time_ms(e0.elapsed_time(e1), dist, device)
+    # end to end: the step's hidden states come from pinned host memory and the reduced output goes back
+    h_host = [h.cpu().pin_memory() for h in hiddens]
+    o_host = [torch.empty((M, cfg.d), dtype=torch.float32).pin_memory() for _ in layers]
+    def step_e2e(i):
+        hiddens[i % n].copy_(h_host[i % n], non_blocking=True)
+        step(i)
+        o_host[i % n].copy_(outs[i % n], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    for i in range(args.warmup):
+        step_e2e(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step_e2e(i)
+    e2e_ms = job_time_ms((time.perf_counter() - t0) * 1e3, dist, device)
+    act = torch.tensor([float(sum(L.get_stats()["n_active"] for L in layers)) / n], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(act)
+    n_active = float(act.item())                 # kept experts with rows, summed over the shards
+    peak, peak_kind = measured_peaks()
+    us = ms_total * 1e3 / args.steps             # the job processes `steps` layers in total
+    layer_bytes = algorithmic_bytes(cfg, M, n_active, 4)
+    agg = layer_bytes / (us * 1e-6) / 1e9
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": us, "unit": "us", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_total / args.steps, "higher_is_better": False, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "parallelism": f"ep{world}: experts split in contiguous blocks, "
+                       "router replicated, one NCCL all-reduce of out[M,d] fp32 per layer inside the timed region",
+                       "l2": f"rotating over {args.copies} independently seeded layer copies", "n_active": n_active},
+            "clocks": clocks,
+            "e2e": {"value": e2e_ms * 1e3 / args.steps, "unit": "us", "h2d_bytes_per_step": h_host[0].numel() * 2,
+                    "d2h_bytes_per_step": o_host[0].numel() * 4},
+            "gpu_launches": layers[0].last_launch_count() * args.steps,
+            "roofline": {"bound": "hbm", "kernel": "ffn_tc_kernel on every rank (its resident kept experts)",
+                         "achieved": agg, "peak": peak * world, "unit": "GB/s", "frac": agg / (peak * world),
+                         "peak_kind": f"of {peak_kind} x {world} GPUs", "traffic": None,
+                         "basis": "algorithmic bytes of the whole layer / step time incl. the all-reduce"},
+            "cpu_baseline": None,
+        }
+        print(json.dumps(line), flush=True)
+    for L in layers:
+        L.destroy()
 
 
 def time_steps(layers, hiddens, outs, k, B, steps, warmup, barrier):
@@ -491,6 +579,8 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="moespec", choices=["moespec", "reference"])
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "ep"],
+                    help="multi-GPU mode: independent replicas (default) or one layer split by experts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true")
     ap.add_argument("--copies", type=int, default=N_COPIES, help="independently seeded layer copies rotated over")
@@ -530,6 +620,11 @@ def main():
 
     if args.tables:
         return run_tables(args, device)
+    if args.mode == "ep":
+        run_expert_parallel(args, dist, device, rank, world, barrier)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
 
     cfg = synth.CONFIGS[WORKLOAD]
     M, k, B = M_TOKENS, cfg.k, B_HEADLINE
@@ -667,6 +762,33 @@ def main():
         for SL in st_layers:
             SL.destroy()
 
+    # expert-parallel shards of the same layers, each timed alone on this GPU: the compute part of an
+    # expert-parallel step is the slowest shard (the all-reduce of out[M,d] is not in these numbers, and no
+    # multi-GPU run is behind them)
+    ep_line = None
+    if not args.no_sweep and world == 1:
+        from paper_2602_16052_b200 import ep as _ep, moespec as _m2
+        ep_line = []
+        for G in (2, 4, 8):
+            per_rank = []
+            for r_ in range(G):
+                first, count = _ep.expert_range(r_, G, cfg.n_experts)
+                sh = []
+                for L0 in layers:
+                    rw, rb, wg, wu, wd = L0._keep
+                    sh.append(_m2.Layer(rw, rb, wg[first:first + count], wu[first:first + count], wd[first:first + count],
+                                        max_M=M, max_k=cfg.k, policy=_m2.SUBSTITUTION, shortlist=_m2.FROM_ALL,
+                                        renormalize=True, out_dtype=out_dtype, resident=(first, count)))
+                n_sh = max(20, args.steps // 8)
+                ms_sh = time_steps(sh, hiddens, outs, k, B, n_sh, 5, barrier)
+                act = sum(L_.get_stats()["n_active"] for L_ in sh) / len(sh)
+                per_rank.append({"rank": r_, "us": ms_sh * 1e3 / n_sh, "n_active": act})
+                for L_ in sh:
+                    L_.destroy()
+            ep_line.append({"shards": G, "slowest_shard_us": max(p_["us"] for p_ in per_rank),
+                            "fastest_shard_us": min(p_["us"] for p_ in per_rank),
+                            "n_active_per_shard": [p_["n_active"] for p_ in per_rank]})
+
     # analysis mode on the same workload: reconstruction error of the three ranking strategies (Section 4.5)
     analysis_line = None
     if not args.no_sweep:
@@ -709,6 +831,7 @@ def main():
             "raw_gating": raw_line,
             "stack": stack_line,
             "analysis": analysis_line,
+            "ep_shards_on_one_gpu": ep_line,
             "fit_time_vs_active_experts": fit,
             "read_stream_GBs_torch_sum": read_stream_gbs,
         }

@@ -86,12 +86,24 @@ typedef struct {
   const void *w_gate;        /* device [N, f, d], d contiguous, 16-byte aligned (W1 of SwiGLU)    */
   const void *w_up;          /* device [N, f, d], d contiguous, 16-byte aligned (W3)              */
   const void *w_down;        /* device [N, d, f], f contiguous, 16-byte aligned (W2)              */
+  /* Expert-parallel shard (the paper ran its largest model on 2 GPUs, Table 3; the experts are the natural
+   * unit to split).  resident_count = 0: this GPU holds all N experts (the default).  Otherwise it holds the
+   * experts resident_first .. resident_first + resident_count - 1 only, and w_gate / w_up / w_down point to
+   * THOSE experts' weights: [resident_count, f, d], [resident_count, f, d], [resident_count, d, f].  The
+   * router (router_w, router_bias) is always the whole [N, d] matrix, so every shard takes the same routing
+   * decisions from the same hidden states without any exchange; a shard runs the expert FFNs of its resident
+   * kept experts only and returns the PARTIAL sum  out_t = sum_{i in A(t), i resident} wgt[t,i] E_i(h_t)
+   * (zeros for a token none of whose kept experts is resident).  The layer output is the sum of the shards'
+   * partial outputs (one all-reduce of [M, d]); out_dtype = MOESPEC_FP32 keeps that sum unrounded.
+   * residual must be 0 on a shard (the caller adds the residual once, after the reduction).               */
+  int resident_first;
+  int resident_count;
 } moespec_layer_desc;
 
 typedef struct {
   int n_union;        /* |E(D)|, Eq. 3                                                            */
   int n_shortlist;    /* |S|                                                                      */
-  int n_active;       /* experts with at least one routed row (what is streamed from HBM)         */
+  int n_active;       /* resident experts with at least one routed row (what is streamed from HBM) */
   int n_rows;         /* R = sum_t |A(t)| routed (token, expert) pairs                            */
   int n_dropped;      /* M*k - R slots that received no expert                                    */
   int status;         /* 0, MOESPEC_ERR_TIMEOUT or MOESPEC_ERR_INTERNAL from the last call        */
@@ -355,7 +367,8 @@ int moespec_reconstruction_error(moespec_layer_t *layer, const void *out_S, cons
 const char *moespec_strerror(int status);
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int moespec_last_cuda_error(void);
-/* major*100 + minor; 110 added the stack, the analysis mode and the early-start FFN kernel. */
+/* major*100 + minor; 110 added the stack, the analysis mode and the early-start FFN kernel;
+ * 120 the expert-parallel shard (resident_first / resident_count at the end of moespec_layer_desc). */
 int moespec_version(void);
 
 #ifdef __cplusplus

@@ -164,6 +164,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.score, N);
   c.take(w.topk_idx, M * K);
   c.take(w.S_rank, N);
+  c.take(w.S_local, N);
   c.take(w.assign_idx, M * K);
   c.take(w.gate_w, M * K);
   c.take(w.count, N);
@@ -248,6 +249,8 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
               const moespec_layer_desc *desc = nullptr) {
   if (!desc) desc = &L->desc;      // the analysis mode runs the same weights under other routing settings
   LaunchCtx c{desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap, stream, 0};
+  c.res_first = L->desc.resident_first;
+  c.res_count = L->desc.resident_count;
   if (L->use_tc) {
     c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
     c.early = tc_early_start(*desc, M) ? 1 : 0;
@@ -326,6 +329,10 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
       d.f > 65536)
     return MOESPEC_ERR_INVALID_ARG;
   if (d.d % 64 || d.f % 64) return MOESPEC_ERR_UNSUPPORTED;
+  if (d.resident_count < 0 || d.resident_first < 0) return MOESPEC_ERR_INVALID_ARG;
+  if (d.resident_count == 0 && d.resident_first != 0) return MOESPEC_ERR_INVALID_ARG;
+  if (d.resident_count > 0 && d.resident_first + d.resident_count > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (d.resident_count > 0 && d.resident_count < d.n_experts && d.residual) return MOESPEC_ERR_INVALID_ARG;
   if (!aligned16(d.router_w) || !aligned16(d.w_gate) || !aligned16(d.w_up) || !aligned16(d.w_down))
     return MOESPEC_ERR_UNSUPPORTED;
   bool use_tc = d.ffn_kernel == MOESPEC_FFN_TENSOR_CORE ||
@@ -346,6 +353,7 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   if (!L) return MOESPEC_ERR_OUT_OF_MEMORY;
   L->magic = kMagic;
   L->desc = d;
+  if (L->desc.resident_count == 0) L->desc.resident_count = d.n_experts;      // all experts are resident
   L->R_cap = d.max_M * d.max_k;
   L->use_tc = use_tc;
   L->arena_bytes = carve(d, L->R_cap, nullptr, nullptr);
@@ -374,7 +382,7 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
   }
   if (use_tc) {
     int cu_res = 0;
-    e = tc_encode_maps(d, L->ws, L->R_cap, &L->maps, &cu_res);
+    e = tc_encode_maps(L->desc, L->ws, L->R_cap, &L->maps, &cu_res);
     if (e == cudaSuccess) e = tc_configure();
     if (e == cudaSuccess) e = routing_configure();
     if (e != cudaSuccess) {
@@ -613,6 +621,8 @@ int moespec_route_from_logits(moespec_layer_t *L, const float *logits, int M, in
   LaunchCtx c{&L->desc, &L->ws, M, k, B > L->desc.n_experts ? L->desc.n_experts : B, L->R_cap,
               static_cast<cudaStream_t>(stream), 0};
   if (L->use_tc) c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
+  c.res_first = L->desc.resident_first;
+  c.res_count = L->desc.resident_count;
   cudaError_t e = launch_route(c, logits);
   if (e != cudaSuccess) return cuda_fail(e);
   L->last_M = M;
@@ -773,7 +783,7 @@ const char *moespec_strerror(int status) {
 }
 
 int moespec_last_cuda_error(void) { return tl_cuda_error; }
-int moespec_version(void) { return 110; }
+int moespec_version(void) { return 120; }
 
 }  // extern "C"
 
@@ -1088,6 +1098,7 @@ int moespec_oracle_ranking(moespec_layer_t *L, const void *hidden, int M, int k,
   const moespec_layer_desc &d = L->desc;
   if (M < 1 || M > d.max_M || k < 1 || k > d.max_k || k > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
   if (n_pick < 1 || n_pick > d.n_experts) return MOESPEC_ERR_INVALID_ARG;
+  if (d.resident_count < d.n_experts) return MOESPEC_ERR_UNSUPPORTED;      // the analysis needs every expert's output
   if (!hidden || !order_host) return MOESPEC_ERR_NULL_POINTER;
   if (!aligned16(hidden) || (out_star && !aligned16(out_star))) return MOESPEC_ERR_UNSUPPORTED;
   if (out_star == hidden) return MOESPEC_ERR_INVALID_ARG;

@@ -44,7 +44,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
                                                       const float *__restrict__ gate_w,
                                                       const int *__restrict__ tokslot2row,
                                                       const T *__restrict__ hidden, TO *__restrict__ out, int d,
-                                                      int k, int residual) {
+                                                      int k, int residual, const int *__restrict__ assign_idx,
+                                                      int res_first, int res_count) {
   const int t = blockIdx.x;
   const int c = (blockIdx.y * blockDim.x + threadIdx.x) * 4;
   __shared__ int s_row[kMaxK];
@@ -52,7 +53,12 @@ __global__ void __launch_bounds__(256) combine_kernel(const float *__restrict__ 
   pdl_trigger();
   pdl_wait();
   if (threadIdx.x < k) {
-    s_row[threadIdx.x] = tokslot2row[(size_t)t * k + threadIdx.x];
+    int row = tokslot2row[(size_t)t * k + threadIdx.x];
+    if (res_count > 0 && row >= 0) {      // expert-parallel shard: only the slots of resident experts
+      const int e = assign_idx[(size_t)t * k + threadIdx.x];
+      if (e < res_first || e >= res_first + res_count) row = -1;
+    }
+    s_row[threadIdx.x] = row;
     s_w[threadIdx.x] = gate_w[(size_t)t * k + threadIdx.x];
   }
   __syncthreads();
@@ -88,7 +94,8 @@ static cudaError_t launch_t(const LaunchCtx &c, const void *hidden, void *out) {
   const moespec_layer_desc &D = *c.desc;
   return launch_kernel(combine_kernel<T, TO>, dim3(c.M, (D.d + 1023) / 1024), dim3(256), 0, c.stream, (const float *)c.ws->y,
                        (const float *)c.ws->gate_w, (const int *)c.ws->tokslot2row, (const T *)hidden, (TO *)out, D.d,
-                       c.k, D.residual);
+                       c.k, D.residual, (const int *)c.ws->assign_idx, c.res_first,
+                       c.res_count > 0 && c.res_count < D.n_experts ? c.res_count : 0);
 }
 
 cudaError_t launch_combine(const LaunchCtx &c, const void *hidden, void *out) {

@@ -21,13 +21,15 @@ __global__ void __launch_bounds__(256) ffn_gateup_cc_kernel(const T *__restrict_
                                                             const T *__restrict__ w_gate,
                                                             const T *__restrict__ w_up, T *__restrict__ h_mid,
                                                             const int *__restrict__ row2expert,
-                                                            const int *__restrict__ counters, int d, int f) {
+                                                            const int *__restrict__ counters, int d, int f,
+                                                            int res_first, int res_count) {
   extern __shared__ float xs[];
   const int r = blockIdx.x;
   pdl_trigger();
   pdl_wait();
   if (r >= counters[2]) return;
-  const int e = row2expert[r];
+  const int e = row2expert[r] - res_first;          // index into the resident experts' weights
+  if (e < 0 || e >= res_count) return;              // another GPU's expert
   const T *x = x_perm + (size_t)r * d;
   for (int j = threadIdx.x; j < d; j += blockDim.x) xs[j] = cc_to_float(x[j]);
   __syncthreads();
@@ -64,13 +66,15 @@ template <typename T>
 __global__ void __launch_bounds__(256) ffn_down_cc_kernel(const T *__restrict__ h_mid,
                                                           const T *__restrict__ w_down, float *__restrict__ y,
                                                           const int *__restrict__ row2expert,
-                                                          const int *__restrict__ counters, int d, int f) {
+                                                          const int *__restrict__ counters, int d, int f,
+                                                          int res_first, int res_count) {
   extern __shared__ float ms[];
   const int r = blockIdx.x;
   pdl_trigger();
   pdl_wait();
   if (r >= counters[2]) return;
-  const int e = row2expert[r];
+  const int e = row2expert[r] - res_first;          // index into the resident experts' weights
+  if (e < 0 || e >= res_count) return;              // another GPU's expert
   const T *m = h_mid + (size_t)r * f;
   for (int j = threadIdx.x; j < f; j += blockDim.x) ms[j] = cc_to_float(m[j]);
   __syncthreads();
@@ -101,12 +105,13 @@ static cudaError_t launch_cc(const LaunchCtx &c, int phase) {
     dim3 g1(rows, (D.f + kColsPerBlock - 1) / kColsPerBlock);
     return launch_kernel(ffn_gateup_cc_kernel<T>, g1, dim3(256), D.d * sizeof(float), c.stream,
                          (const T *)c.ws->x_perm, (const T *)D.w_gate, (const T *)D.w_up, (T *)c.ws->h_mid,
-                         (const int *)c.ws->row2expert, (const int *)c.ws->counters, D.d, D.f);
+                         (const int *)c.ws->row2expert, (const int *)c.ws->counters, D.d, D.f, c.res_first,
+                         c.res_count > 0 ? c.res_count : D.n_experts);
   } else {
     dim3 g2(rows, (D.d + kColsPerBlock - 1) / kColsPerBlock);
     return launch_kernel(ffn_down_cc_kernel<T>, g2, dim3(256), D.f * sizeof(float), c.stream,
                          (const T *)c.ws->h_mid, (const T *)D.w_down, c.ws->y, (const int *)c.ws->row2expert,
-                         (const int *)c.ws->counters, D.d, D.f);
+                         (const int *)c.ws->counters, D.d, D.f, c.res_first, c.res_count > 0 ? c.res_count : D.n_experts);
   }
 }
 

@@ -110,7 +110,9 @@ struct TcArgs {
   // early start (see the kernel's header comment)
   int early;                 // 1: tickets below the grid size are started on before routing has finished
   const int *early_flag;     // 0 until the routing kernel has published the shortlist, then |S| + 1
-  const int *S_rank;         // shortlist in rank order
+  const int *S_rank;         // the resident part of the shortlist in rank order
+  int res_first, res_count;  // experts whose weights this GPU holds: the weight tensors start at expert res_first
+  const int *assign_idx;     // [M, k] kept expert per slot (the combine of a shard skips slots of other GPUs' experts)
   const int *perm_row2tok;   // gather order: row -> token
   int tiles_real;            // f / ru: gate/up units per expert
   int static_nS;             // > 0: fixed shortlist (Eq. 4) of this size, known before any kernel of the call runs
@@ -430,7 +432,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
           const int j = phase == 0 ? (lane >> 1) : lane;
           const int col = (kc * cps + j) * kChunkK;
           const CUtensorMap *mw = phase == 0 ? ((lane & 1) ? &maps.w_up : &maps.w_gate) : &maps.w_down;
-          tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * ru, expert, wpol);
+          tma_load_3d(stage + lane * sub_bytes, mw, full, col, tile * ru, expert - a.res_first, wpol);
         }
       };
       auto rows = [&](int kc) {
@@ -679,10 +681,17 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   const int warps_total = (kThreads / 32) * (int)gridDim.x;
   int my_row = -1;
   float my_w = 0.f;
+  // an expert-parallel shard adds up the slots of its resident experts only (the other rows of y are not its own)
+  const bool shard = a.res_count > 0;
+  auto resident_slot = [&](int t, int slot) {
+    const int e = a.assign_idx[(size_t)t * k + slot];
+    return e >= a.res_first && e < a.res_first + a.res_count;
+  };
   if (warp_global < n_items && lane < k) {
     const int t = warp_global / slices;
     my_row = a.tokslot2row[(size_t)t * k + lane];
     my_w = a.gate_w[(size_t)t * k + lane];
+    if (shard && my_row >= 0 && !resident_slot(t, lane)) my_row = -1;
   }
   if (threadIdx.x == 0 && !*abort_flag) {
     const int n_down = a.n_units[1];
@@ -702,6 +711,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     if (item != warp_global) {                               // later items: this token's slots
       my_row = lane < k ? a.tokslot2row[(size_t)t * k + lane] : -1;
       my_w = lane < k ? a.gate_w[(size_t)t * k + lane] : 0.f;
+      if (shard && my_row >= 0 && !resident_slot(t, lane)) my_row = -1;
     }
     {
       float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -788,7 +798,7 @@ cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int
   const CUtensorMapDataType tm_dtype =
       d.dtype == MOESPEC_FP16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
   auto weights = [&](CUtensorMap *m, const void *base, int rows, int K, int box_rows) -> CUresult {
-    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)d.n_experts};
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)(d.resident_count > 0 ? d.resident_count : d.n_experts)};
     cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)rows * K * 2};
     cuuint32_t box[3] = {kChunkK, (cuuint32_t)box_rows, 1};
     return enc(m, tm_dtype, 3, const_cast<void *>(base), dims, strides, box, ones,
@@ -848,6 +858,7 @@ int tc_rows_per_unit(const moespec_layer_desc &D, int M, int k, int B) {
   // shorter slabs double the L2->SM traffic per weight byte); 64-row slabs only pay off when there would
   // otherwise be fewer gate/up units than half the SMs (a handful of kept experts, e.g. M = 1).
   int active = B < D.n_experts ? B : D.n_experts;          // upper bound of kept experts that get rows
+  if (D.resident_count > 0 && D.resident_count < active) active = D.resident_count;      // ... on this GPU
   if ((long long)M * k < active) active = M * k;
   static const int forced = [] { const char *v = experiment_env("MOESPEC_FORCE_RU"); return v ? atoi(v) : 0; }();
   if (forced == 128 || forced == 64 || forced == 32) return forced;     // experiments only
@@ -900,7 +911,10 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.out_is_fp32 = (D.out_dtype ? D.out_dtype : D.dtype) == MOESPEC_FP32;
   a.early = c.early;
   a.early_flag = c.ws->early_flag;
-  a.S_rank = c.ws->S_rank;
+  a.S_rank = c.ws->S_local;
+  a.res_first = c.res_first;
+  a.res_count = c.res_count > 0 && c.res_count < D.n_experts ? c.res_count : 0;      // 0: not a shard
+  a.assign_idx = c.ws->assign_idx;
   a.perm_row2tok = c.ws->perm_row2tok;
   a.tiles_real = D.f / ru;
   a.static_nS = 0;

@@ -52,6 +52,7 @@ struct Workspace {
   double *score;        // [N]
   int *topk_idx;        // [max_M, max_k]
   int *S_rank;          // [N]
+  int *S_local;         // [N] the resident members of the shortlist in rank order (what the FFN kernel starts on)
   int *assign_idx;      // [max_M, max_k]
   float *gate_w;        // [max_M, max_k]
   int *count;           // [N]
@@ -95,6 +96,7 @@ struct LaunchCtx {
   cudaStream_t stream;
   int ru;               // weight rows per tensor-core work unit for this call (0: CUDA-core path)
   int early = 0;        // 1: the FFN kernel starts on the shortlist before routing has finished (see ffn_tc.cu)
+  int res_first = 0, res_count = 0; // resident experts [res_first, res_first + res_count) (res_count = N: all)
   long long debug_spin_limit = 0;   // test hook: bound of device-side waits in cycles (0 = default)
   int debug_ready_bias = 0;         // test hook: extra slabs every down unit waits for (never reported)
 };

@@ -480,6 +480,7 @@ struct RouteArgs {
   int early;                    // the FFN kernel starts on the shortlist before this kernel has finished
   int ffn_ctas;                 // CTAs of the FFN kernel: CTA c starts on gate/up unit c of the list
   int rows_later;               // the row of every (token, slot) pair is left to the row kernel (large trees)
+  int res_first, res_count;     // experts resident on this GPU (expert-parallel shard); res_count = N: all
 };
 
 constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
@@ -667,10 +668,34 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     if (lane == 0) s_Smask[warp] = word;
   }
   __syncthreads();
-  // publish the shortlist (S_rank was written by this CTA's threads before the barrier): the FFN kernel's
+  // What the FFN kernel works on is the part of the shortlist that is resident on this GPU, in rank order
+  // (all of it unless this layer is an expert-parallel shard): s_Srank / nS_l from here on.  The shortlist
+  // itself stays in s_Smask (re-routing) and in ws.S_rank.
+  const bool shard = a.res_count < N;
+  int nS_l = nS;
+  if (shard) {
+    int e_r = 0;
+    bool res = false;
+    if (tid < nS) {
+      e_r = s_Srank[tid];
+      res = e_r >= a.res_first && e_r < a.res_first + a.res_count;
+    }
+    const unsigned bal = __ballot_sync(kFull, res);
+    if (lane == 0) s_warp_tot[warp] = (unsigned long long)__popc(bal);
+    __syncthreads();                         // every thread has read its entry of s_Srank
+    int pos = __popc(bal & ((1u << lane) - 1u));
+    for (int w = 0; w < warp; ++w) pos += (int)s_warp_tot[w];
+    nS_l = 0;
+    for (int w = 0; w < kRouteWarps; ++w) nS_l += (int)s_warp_tot[w];
+    if (res) s_Srank[pos] = e_r;
+    __syncthreads();
+  }
+  if (blockIdx.x == 0 && ws.S_local && tid < nS_l) ws.S_local[tid] = s_Srank[tid];
+  __syncthreads();
+  // publish the shortlist (S_local was written by this CTA's threads before the barrier): the FFN kernel's
   // CTAs start streaming the weights of its best-ranked experts while the rest of the routing runs
-  if (blockIdx.x == 0 && tid == 0 && ws.early_flag)      // the barrier above orders the other threads' S_rank stores before this release
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag), "r"(nS + 1) : "memory");
+  if (blockIdx.x == 0 && tid == 0 && ws.early_flag)      // the barrier above orders the other threads' stores before this release
+    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag), "r"(nS_l + 1) : "memory");
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
@@ -693,10 +718,12 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     const int c = tid < N ? __ldcg(ws.count_acc + tid) : 0;
     if (cm_cached)
       for (int i = tid; i < N * used_words; i += blockDim.x) s_colmask[i] = __ldcg(ws.colmask + i);
-    const int chunks = (c + kMaxTokChunk - 1) / kMaxTokChunk;
+    // work units and the active count cover the resident experts only; rows and offsets cover all
+    const bool resident = tid >= a.res_first && tid < a.res_first + a.res_count;
+    const int chunks = resident ? (c + kMaxTokChunk - 1) / kMaxTokChunk : 0;
     // rows in bits 0..23, chunks in bits 24..43, active flag in bits 44..
     const unsigned long long v = (unsigned long long)c | ((unsigned long long)chunks << 24) |
-                                 ((unsigned long long)(c > 0) << 44);
+                                 ((unsigned long long)(c > 0 && resident) << 44);
     unsigned long long inc = v;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -715,13 +742,13 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       ws.count[tid] = c;
       ws.offset[tid] = row0;
       ws.score[tid] = (double)s_fx[tid] * (1.0 / kScoreScale);
-      if (c > 0) ws.active[ai] = tid;
+      if (c > 0 && resident) ws.active[ai] = tid;
       for (int cc = 0; cc < chunks && ub + cc < 2 * kMaxExperts; ++cc) s_chunk_expert[ub + cc] = tid;
       if (tid == N - 1) {
         s_offset[N] = row0 + c;
         ws.offset[N] = row0 + c;
         s_unit_base[N] = ub + chunks;
-        s_nactive = ai + (c > 0);
+        s_nactive = ai + (c > 0 && resident);
       }
     }
   }
@@ -730,10 +757,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     // Early start (M <= 128, so an expert has at most one token chunk): the unit list follows the
     // shortlist's rank order, and the experts whose gate/up units the FFN kernel's CTAs start on before
     // this list exists (CTA c takes unit c) keep their place even if no token was routed to them.
-    const int n_head = min((a.ffn_ctas + a.tiles_up - 1) / a.tiles_up, nS);
+    const int n_head = min((a.ffn_ctas + a.tiles_up - 1) / a.tiles_up, nS_l);
     bool present = false;
     int e_r = 0;
-    if (tid < nS) {
+    if (tid < nS_l) {
       e_r = s_Srank[tid];
       present = s_count[e_r] > 0 || tid < n_head;
     }
@@ -830,7 +857,8 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       }
     }
   } else if (warp == 7) {
-    for (int r = lane; r < nS; r += 32) cov += (double)s_fx[s_Srank[r]];
+    for (int e = lane; e < N; e += 32)
+      if ((s_Smask[e >> 5] >> (e & 31)) & 1u) cov += (double)s_fx[e];
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cov += shfl_xor_double(cov, o);
     cov *= 1.0 / kScoreScale;
@@ -880,6 +908,8 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.early = c.ru > 0 ? c.early : 0;
   a.ffn_ctas = tc_grid_size(D.device);
   a.rows_later = rows_in_row_kernel(c.M);
+  a.res_first = c.res_count > 0 ? c.res_first : 0;
+  a.res_count = c.res_count > 0 ? c.res_count : D.n_experts;
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);
   if (a.N <= 32) return launch_kernel(route_kernel<1>, grid, block, 0, c.stream, a);
   if (a.N <= 64) return launch_kernel(route_kernel<2>, grid, block, 0, c.stream, a);

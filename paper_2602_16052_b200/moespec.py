@@ -46,6 +46,7 @@ class LayerDesc(C.Structure):
         ("residual", C.c_int), ("ffn_kernel", C.c_int), ("device", C.c_int),
         ("router_w", C.c_void_p), ("router_bias", C.c_void_p),
         ("w_gate", C.c_void_p), ("w_up", C.c_void_p), ("w_down", C.c_void_p),
+        ("resident_first", C.c_int), ("resident_count", C.c_int),
     ]
 
 
@@ -166,14 +167,19 @@ class Layer:
 
     def __init__(self, router_w, router_bias, w_gate, w_up, w_down, *, max_M: int, max_k: int,
                  policy: int = SUBSTITUTION, shortlist: int = FROM_ALL, renormalize: bool = True,
-                 residual: bool = False, ffn_kernel: int = FFN_AUTO, out_dtype: Optional[torch.dtype] = None):
+                 residual: bool = False, ffn_kernel: int = FFN_AUTO, out_dtype: Optional[torch.dtype] = None,
+                 resident: Optional[tuple] = None):
+        """resident = (first, count): this layer is an expert-parallel shard that holds the experts
+        first .. first+count-1 only; w_gate / w_up / w_down are then THOSE experts' weights ([count, ...]) and
+        verify_layer returns the shard's partial sum.  None: all N experts are here."""
         for t in (router_w, w_gate, w_up, w_down):
             if not (t.is_cuda and t.is_contiguous()):
                 raise ValueError("weights must be contiguous CUDA tensors")
         N, d = router_w.shape
         f = w_gate.shape[1]
-        if tuple(w_gate.shape) != (N, f, d) or tuple(w_up.shape) != (N, f, d) or tuple(w_down.shape) != (N, d, f):
-            raise ValueError("weight shapes must be [N,f,d], [N,f,d], [N,d,f]")
+        E = N if resident is None else int(resident[1])
+        if tuple(w_gate.shape) != (E, f, d) or tuple(w_up.shape) != (E, f, d) or tuple(w_down.shape) != (E, d, f):
+            raise ValueError("weight shapes must be [E,f,d], [E,f,d], [E,d,f] with E the experts held here")
         dt = _DTYPES[router_w.dtype]
         if router_bias is not None:
             router_bias = router_bias.to(device=router_w.device, dtype=torch.float32).contiguous()
@@ -188,7 +194,9 @@ class Layer:
                          ffn_kernel=ffn_kernel, device=router_w.device.index or 0,
                          router_w=router_w.data_ptr(),
                          router_bias=None if router_bias is None else router_bias.data_ptr(),
-                         w_gate=w_gate.data_ptr(), w_up=w_up.data_ptr(), w_down=w_down.data_ptr())
+                         w_gate=w_gate.data_ptr(), w_up=w_up.data_ptr(), w_down=w_down.data_ptr(),
+                         resident_first=0 if resident is None else int(resident[0]),
+                         resident_count=0 if resident is None else int(resident[1]))
         h = C.c_void_p()
         _check(lib().moespec_layer_create(C.byref(desc), C.byref(h)), "moespec_layer_create")
         self._h = h
