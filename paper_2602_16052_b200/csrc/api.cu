@@ -164,7 +164,6 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.score, N);
   c.take(w.topk_idx, M * K);
   c.take(w.S_rank, N);
-  c.take(w.S_local, N);
   c.take(w.assign_idx, M * K);
   c.take(w.gate_w, M * K);
   c.take(w.count, N);
@@ -180,7 +179,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.colmask, N * (size_t)w.mask_words);
   c.take(w.arrive, M);
   c.take(w.arrive_route, 4);
-  c.take(w.early_flag, 4);
+  c.take(w.early_flag, N);
   c.take(w.calib_count, N);
   c.take(w.static_pos, N);
   c.take(w.static_order, N);

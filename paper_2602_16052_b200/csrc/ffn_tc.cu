@@ -109,8 +109,9 @@ struct TcArgs {
   long long spin_limit; // cycles after which any wait gives up
   // early start (see the kernel's header comment)
   int early;                 // 1: tickets below the grid size are started on before routing has finished
-  const int *early_flag;     // 0 until the routing kernel has published the shortlist, then |S| + 1
-  const int *S_rank;         // the resident part of the shortlist in rank order
+  const int *early_flag;     // [n_words] word r: 0 until the routing kernel has published the shortlist, then the
+                             // resident expert of rank r, plus one, or -1 when there are fewer
+  int n_words;
   int res_first, res_count;  // experts whose weights this GPU holds: the weight tensors start at expert res_first
   const int *assign_idx;     // [M, k] kept expert per slot (the combine of a shard skips slots of other GPUs' experts)
   const int *perm_row2tok;   // gather order: row -> token
@@ -332,18 +333,20 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       // keeps the routed tokens only.  The routing kernel builds the unit list in the same order and keeps
       // the experts of those ranks in it even without rows, so unit c of the list is this unit.
       if (lane == 0 && t_first < (int)gridDim.x) {
-        int fl = a.static_nS + 1;        // a fixed shortlist needs no publication: stream from the first cycle
-        const int *rank = a.static_nS > 0 ? a.static_order : a.S_rank;
-        if (a.static_nS == 0) {
+        const int r = t_first / a.tiles_real;
+        int v = -1;                      // the expert of rank r, plus one
+        if (a.static_nS > 0) {           // a fixed shortlist needs no publication: stream from the first cycle
+          if (r < a.static_nS) v = a.static_order[r] + 1;
+        } else if (r < a.n_words) {
           const long long t0 = clock64();
-          while ((fl = ld_acquire(a.early_flag)) == 0) {
+          while ((v = ld_acquire(a.early_flag + r)) == 0) {
             if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
             __nanosleep(32);
           }
         }
-        if (ok && t_first < (fl - 1) * a.tiles_real) {
-          un.expert = __ldcg(rank + t_first / a.tiles_real);
-          un.tile = t_first % a.tiles_real;
+        if (ok && v > 0) {
+          un.expert = v - 1;
+          un.tile = t_first - r * a.tiles_real;
           un.n_rows = a.M;
           un.pad0 = 1;                 // dense: every token, rows of `hidden`
           un.pad1 = t_first;           // its place in the unit list
@@ -911,7 +914,7 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.out_is_fp32 = (D.out_dtype ? D.out_dtype : D.dtype) == MOESPEC_FP32;
   a.early = c.early;
   a.early_flag = c.ws->early_flag;
-  a.S_rank = c.ws->S_local;
+  a.n_words = D.n_experts;
   a.res_first = c.res_first;
   a.res_count = c.res_count > 0 && c.res_count < D.n_experts ? c.res_count : 0;      // 0: not a shard
   a.assign_idx = c.ws->assign_idx;

@@ -52,7 +52,6 @@ struct Workspace {
   double *score;        // [N]
   int *topk_idx;        // [max_M, max_k]
   int *S_rank;          // [N]
-  int *S_local;         // [N] the resident members of the shortlist in rank order (what the FFN kernel starts on)
   int *assign_idx;      // [max_M, max_k]
   float *gate_w;        // [max_M, max_k]
   int *count;           // [N]
@@ -69,7 +68,8 @@ struct Workspace {
   unsigned *colmask;    // [N, ceil(max_M/32)] bit t of row i: expert i in A(t)
   int *arrive;          // [max_M] arrival counters of router_topk_kernel's token tiles
   int *arrive_route;    // [1] arrival counter of route_kernel's CTAs
-  int *early_flag;      // [1] 0 until the shortlist of the call is published, then |S| + 1 (may be null)
+  int *early_flag;      // [N] word r is 0 until the shortlist of the call is published, then (resident expert of
+                        // rank r) + 1, or -1 when there are fewer (may be null)
   int mask_words;       // ceil(max_M / 32)
   long long *calib_count;   // [N] Eq. 4 calibration counts c_i
   int *static_pos;          // [N] position of expert i in the fixed ordering (INT_MAX: not listed)

@@ -155,21 +155,23 @@ __device__ __forceinline__ void clear_colmask(unsigned *colmask, int words) {
   for (int i = cta * blockDim.x + threadIdx.x; i < words; i += n_cta * blockDim.x) colmask[i] = 0u;
 }
 
-// The FFN kernel's control words must be in their initial state when its first CTA starts: the shortlist flag
-// at 0 (the routing kernel publishes the call's shortlist later; the FFN kernel polls the flag), its unit
+// The FFN kernel's control words must be in their initial state when its first CTA starts: the shortlist words
+// at 0 (the routing kernel publishes the call's shortlist later; the FFN kernel's CTAs poll them), its unit
 // dispenser and its down-unit counter at 0.  The router kernel's first CTA sets them: it runs after the
 // previous call's FFN kernel has completed (it has just waited for that) and completes before this call's FFN
 // kernel can start -- except with a fixed shortlist, where the FFN kernel is released right behind this kernel's
 // CTAs: there the stores are performed (fence) before this CTA releases the dependents.
-__device__ __forceinline__ void reset_ffn_control(int *early_flag, int *unit_counter, int fence_reset) {
+__device__ __forceinline__ void reset_ffn_control(int *early_flag, int n_words, int *unit_counter, int fence_reset) {
   if (!early_flag || blockIdx.x != 0 || blockIdx.y != 0) return;
+  for (int i = threadIdx.x; i < n_words; i += blockDim.x) early_flag[i] = 0;
   if (threadIdx.x == 0) {
-    *early_flag = 0;
     unit_counter[0] = 0;
     unit_counter[1] = 0;
-    if (fence_reset) __threadfence();
   }
-  if (fence_reset) __syncthreads();
+  if (fence_reset) {
+    __threadfence();
+    __syncthreads();
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -203,7 +205,7 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       if ((lane + u * 32) * VEC < d) rw[u] = *reinterpret_cast<const uint4 *>(Wr + (size_t)i * d + (lane + u * 32) * VEC);
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
-  reset_ffn_control(early_flag, unit_counter, fence_reset);
+  reset_ffn_control(early_flag, N, unit_counter, fence_reset);
   // Dependents are released only now: with a fixed shortlist the FFN kernel of this call starts at once,
   // and it reads `hidden`, which the previous kernel in the stream may have produced.
   pdl_trigger();
@@ -330,7 +332,7 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
     }
   }
   pdl_wait();          // hidden may be the previous layer's output; the workspace is still in use until then
-  reset_ffn_control(early_flag, unit_counter, fence_reset);
+  reset_ffn_control(early_flag, N, unit_counter, fence_reset);
   pdl_trigger();       // released only now: see router_topk_kernel
   clear_colmask(colmask, N * ((M + 31) >> 5));
   const T *hb = hidden + (size_t)min(t0 + g, M - 1) * d + warp * kw + tg * 8;
@@ -450,7 +452,8 @@ __global__ void __launch_bounds__(128) softmax_topk_kernel(const float *logits, 
   const int t = blockIdx.x * 4 + (threadIdx.x >> 5);
   pdl_trigger();
   pdl_wait();
-  if (early_flag && blockIdx.x == 0 && threadIdx.x == 0) *early_flag = 0;
+  if (early_flag && blockIdx.x == 0)
+    for (int i = threadIdx.x; i < N; i += blockDim.x) early_flag[i] = 0;
   clear_colmask(colmask, N * ((M + 31) >> 5));
   if (t < M)
     token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt,
@@ -690,12 +693,13 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     if (res) s_Srank[pos] = e_r;
     __syncthreads();
   }
-  if (blockIdx.x == 0 && ws.S_local && tid < nS_l) ws.S_local[tid] = s_Srank[tid];
-  __syncthreads();
-  // publish the shortlist (S_local was written by this CTA's threads before the barrier): the FFN kernel's
-  // CTAs start streaming the weights of its best-ranked experts while the rest of the routing runs
-  if (blockIdx.x == 0 && tid == 0 && ws.early_flag)      // the barrier above orders the other threads' stores before this release
-    asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag), "r"(nS_l + 1) : "memory");
+  // publish the shortlist: the FFN kernel's CTAs start streaming the weights of its best-ranked experts while
+  // the rest of the routing runs.  One word per rank (the expert, plus one; -1 beyond the last one): a CTA
+  // polls the word of the rank it starts on and needs nothing else, so each word is its own payload and a
+  // relaxed store suffices.
+  if (blockIdx.x == 0 && ws.early_flag && tid < N)
+    asm volatile("st.relaxed.gpu.global.s32 [%0], %1;" ::"l"(ws.early_flag + tid), "r"(tid < nS_l ? s_Srank[tid] + 1 : -1)
+                 : "memory");
 
   // ---- re-routing (Eq. 7 / Eq. 8) and mixing weights (Section 3.3) of this warp's token
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
