@@ -410,9 +410,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       const int draw_at = k_iters > 6 ? k_iters - 6 : 0;
       const int chunk = __shfl_sync(0xffffffffu, un.chunk, 0);
       // A stage is armed and its weight copies issued by head(); its token-row copies by rows().  A down
-      // unit reads h_mid, which is complete only when every gate/up slab of its expert has been published:
-      // its first stages' weights are therefore requested BEFORE that wait, so that a CTA that runs into
-      // the dependency keeps streaming instead of idling.
+      // unit reads h_mid, which is complete only when every gate/up slab of its expert has been published.
       int armed = 0;                                // stages of this unit whose barrier has been armed
       auto head = [&](int kc) {
         const uint32_t s = (it + kc) % n_stages, ph = ((it + kc) / n_stages) & 1u;
@@ -450,19 +448,40 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       };
       int n_pre = 0;
       if (phase == 1) {
-        n_pre = k_iters < n_stages ? k_iters : n_stages;
-        for (int kc = 0; kc < n_pre && ok; ++kc) head(kc);
-        if (ok && lane == 0) {
-          const long long t0 = clock64();
-          while (ld_acquire(a.ready + chunk) < a.tiles_up) {
-            if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
-            __nanosleep(64);
-          }
+        // Usually the expert's slabs were published long ago.  The counter is read while the slot of the
+        // first stage drains behind the previous unit; if it is complete, this unit's stages follow the
+        // previous unit's without a gap, weights and rows together.  (Requesting the weights of several
+        // stages first, then looking at the counter, then requesting the rows left the ring standing still
+        // for two round trips at the start of every down unit.)
+        int seen = 0;
+        if (lane == 0) seen = ld_acquire(a.ready + chunk);
+        head(0);
+        int is_ready = 0;
+        if (ok && lane == 0 && seen >= a.tiles_up) {
+          is_ready = 1;
           fence_proxy_async();                      // order the acquire before the TMA reads of h_mid
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        // on an abort the armed stages still receive their weight copies; the drain below waits for them
-        for (int kc = 0; kc < n_pre && ok; ++kc) rows(kc);
+        is_ready = __shfl_sync(0xffffffffu, is_ready, 0);
+        if (ok && is_ready) {
+          rows(0);
+          n_pre = 1;
+        } else if (ok) {
+          // not yet: the weights of the first stages are requested BEFORE the wait, so that a CTA that runs
+          // into the dependency keeps streaming instead of idling
+          n_pre = k_iters < n_stages ? k_iters : n_stages;
+          for (int kc = 1; kc < n_pre && ok; ++kc) head(kc);
+          if (ok && lane == 0) {
+            const long long t0 = clock64();
+            while (ld_acquire(a.ready + chunk) < a.tiles_up) {
+              if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
+              __nanosleep(64);
+            }
+            fence_proxy_async();
+          }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          // on an abort the armed stages still receive their weight copies; the drain below waits for them
+          for (int kc = 0; kc < n_pre && ok; ++kc) rows(kc);
+        }
       }
       for (int kc = n_pre; kc < k_iters && ok; ++kc) {
         head(kc);
