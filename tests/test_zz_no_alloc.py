@@ -86,6 +86,32 @@ def test_route_static_large_tree_against_the_oracle():
         assert n_act == len(r["active"]) and R == len(r["perm_row2tok"])
 
 
+def test_route_static_replayed_from_a_captured_graph():
+    """One of the callers this entry point is for runs inside a stream capture.  The first call on the device is
+    made outside the capture (it looks up the scratch array's address); a later call is then captured into a
+    CUDA graph and the graph is replayed on new logits: every replay must give the handle-based results."""
+    from paper_2602_16052_b200 import moespec as m
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = synth.gen_layer(cfg, 23, 0, "cuda")
+    k, M, B = cfg.k, 200, 20
+    mk_logits = lambda seed: (synth.gen_hidden(cfg, M, seed, 0, "cuda").float() @ case["router_w"].float().T
+                              + case["router_bias"]).contiguous()
+    z = mk_logits(23)
+    out = m.route_static(z, k, B, m.SUBSTITUTION, m.FROM_ALL, True)           # first call: outside any capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        m.route_static(z, k, B, m.SUBSTITUTION, m.FROM_ALL, True, out=out, stream=torch.cuda.current_stream())
+    for seed in (24, 25):
+        z.copy_(mk_logits(seed))
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        want = reference_routing(m, case, z, k, B, m.SUBSTITUTION, m.FROM_ALL, True)
+        check_same(out, want, M, k)
+
+
 def test_route_static_rejects_sizes_beyond_its_scratch():
     from paper_2602_16052_b200 import moespec as m
     z = torch.zeros((m.ROUTE_STATIC_MAX_M + 1, 8), dtype=torch.float32, device="cuda")
