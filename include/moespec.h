@@ -123,7 +123,9 @@ int moespec_layer_create(const moespec_layer_desc *desc, moespec_layer_t **out_l
  * no kept expert when residual = 0).  out must not alias hidden.
  * stream: a cudaStream_t (NULL = default stream).  Enqueues and returns.
  * A handle owns one workspace: calls on the same handle must be ordered (same
- * stream, or synchronised by the caller); different handles are independent.
+ * stream, or synchronised by the caller); different handles are independent and
+ * their calls may overlap on the GPU (no kernel of the layer needs its whole grid
+ * to be resident at once).
  * The call may be captured into a CUDA graph by the caller (it allocates nothing
  * and only enqueues kernels).
  * Errors: BAD_HANDLE, NULL_POINTER, INVALID_ARG, CUDA (launch failure). */
@@ -134,7 +136,9 @@ int moespec_verify_layer(moespec_layer_t *layer, const void *hidden, int M, int 
  * runs the layer, delivers the result in out (host [M, d], out_dtype) and synchronises
  * before returning.  With pinned (page-locked) buffers the whole step is captured
  * once per (M, k, B, buffer pair) into a CUDA graph and replayed with one launch on
- * an internal stream, after the work already queued on `stream`.  When the pinned buffers
+ * an internal stream, after the work already queued on `stream`; the handle keeps the
+ * four most recently used instantiations, so a caller may alternate between a few
+ * trees or buffer pairs without re-capturing.  When the pinned buffers
  * are mapped into the device's address space (the default under unified addressing)
  * the graph has no copy nodes: a kernel pulls hidden over the interconnect into a
  * staging buffer and the layer's last kernel writes out directly to the host buffer.
@@ -286,10 +290,10 @@ int moespec_destroy(moespec_layer_t *layer);
  * per (M, k, budgets, buffer pair) on an internal stream with programmatic
  * dependent launch edges, so that each kernel's prologue (barrier set-up, tensor
  * memory allocation, the router-matrix prefetch of the next layer) overlaps the
- * tail of its predecessor; the cached graph is re-instantiated when an argument
- * or a layer setting (static ranking, profiling, wait bounds) changes.  The first
- * call with new arguments therefore allocates (graph instantiation); later calls
- * do not.  moespec_stack_set_graph(stack, 0) enqueues the kernels one by one
+ * tail of its predecessor; the four most recently used instantiations are kept, and
+ * one is re-made when a layer setting (static ranking, profiling, wait bounds)
+ * changes.  The first call with new arguments therefore allocates (graph
+ * instantiation); later calls do not.  moespec_stack_set_graph(stack, 0) enqueues the kernels one by one
  * instead (same results). */
 typedef struct moespec_stack moespec_stack_t;
 

@@ -492,7 +492,8 @@ def test_bounded_wait_expires_cleanly_and_layer_recovers():
 
 
 # ------------------------------------------------------------------ full Mixtral-shaped layer, sampled tokens
-@pytest.mark.parametrize("M,B,ffn", [(15, 4, "tensor_core"), (63, 6, "tensor_core"), (63, 8, "tensor_core"),
+@pytest.mark.parametrize("M,B,ffn", [(15, 4, "tensor_core"), (15, 6, "tensor_core"), (15, 8, "tensor_core"),
+                                     (63, 4, "tensor_core"), (63, 6, "tensor_core"), (63, 8, "tensor_core"),
                                      (15, 4, "cuda_core")])
 def test_mixtral_full_shape_sampled_tokens(M, B, ffn):
     """d=4096, f=14336, N=8, k=2 at full size.  Routing is checked for every token; layer outputs are

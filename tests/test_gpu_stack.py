@@ -112,11 +112,11 @@ def test_stack_at_full_layer_size():
 
 def test_wide_router_stack_at_full_layer_size():
     """Three layers of the 48-layer Qwen3-30B-A3B-shaped stack at full size (d=2048, N=128, k=8, f=768),
-    renormalised gating and one graph launch per pass as the benchmark tables run it, at three points of its
+    renormalised gating and one graph launch per pass as the benchmark tables run it, at all six points of its
     (M, B) sweep; each layer checked against the oracle on the GPU's own input to that layer."""
     cfg = synth.CONFIGS["qwen3"].with_(n_layers=3)
     cases, layers, stack = build_stack(cfg, 127, seed=2000)
-    for M, B in ((63, 32), (63, 64), (127, 128)):
+    for M, B in ((63, 32), (63, 64), (63, 128), (127, 32), (127, 64), (127, 128)):
         x0 = synth.gen_hidden(cfg, M, seed=2000, device="cuda")
         out = stack.verify_stack(x0, cfg.k, B)
         torch.cuda.synchronize()
