@@ -281,15 +281,16 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
 
 // ---------------------------------------------------------------------------
 // K1 for larger trees: the same logits, softmax and top-k, with the dot products on the tensor cores.
-// A CTA takes 16 experts x 8 tokens; its eight warps split K, each running m16n8k16 MMAs (experts on the
+// A CTA takes 16 experts x 8 tokens; its NW (sixteen, or eight) warps split K, each running m16n8k16 MMAs (experts on the
 // M axis, tokens on the N axis) on operands loaded straight from global memory: thread (g, tg) of a warp
 // reads 16 contiguous bytes of router rows g and g+8 and of token row g at K offset 32*step + 8*tg and
 // feeds them to two MMAs.  That assigns memory positions to the instruction's k slots in a permuted
 // order, which is immaterial for a dot product as long as both operands use the same one.  The warps'
 // partial tiles meet in shared memory and are added in warp order (a fixed order: logits are
 // reproducible), then the kernel ends like router_topk_kernel: arrival counter per token tile, softmax
-// and top-k by the CTA that completes the tile.  The CUDA-core kernel above spends its time converting and
-// multiplying element by element, which is what limits it beyond ~64 tokens.
+// and top-k by the CTA that completes the tile (with sixteen warps the two run on separate warps per token).
+// The CUDA-core kernel above spends its time converting and multiplying element by element, which is what
+// limits it beyond ~64 tokens.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                           uint32_t b1, __nv_bfloat16) {
@@ -306,8 +307,8 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
 
 constexpr int kRmExperts = 16, kRmTokens = 8, kRmSteps = 8;     // tile of a CTA; 32-element K steps per batch
 
-template <typename T>
-__global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
+template <typename T, int NW>
+__global__ void __launch_bounds__(NW * 32) router_mma_kernel(const T *__restrict__ hidden, const T *__restrict__ Wr,
                                                          const float *__restrict__ bias, float *logits, double *prob,
                                                          int *topk_idx, unsigned long long *score_fx, int *natcnt,
                                                          int *arrive, int *early_flag, int *unit_counter,
@@ -316,9 +317,9 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int g = lane >> 2, tg = lane & 3;
   const int e0 = blockIdx.x * kRmExperts, t0 = blockIdx.y * kRmTokens;
-  __shared__ float s_part[8][kRmExperts * kRmTokens];
+  __shared__ float s_part[NW][kRmExperts * kRmTokens];
   __shared__ int s_last;
-  const int kw = d / 8;                                   // K range of this warp: [warp*kw, warp*kw + kw)
+  const int kw = d / NW;                                  // K range of this warp: [warp*kw, warp*kw + kw)
   const int ra = min(e0 + g, N - 1), rb = min(e0 + g + 8, N - 1);      // clamped: rows beyond N are never stored
   const T *wa = Wr + (size_t)ra * d + warp * kw + tg * 8;
   const T *wb = Wr + (size_t)rb * d + warp * kw + tg * 8;
@@ -367,7 +368,7 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
     const int el = threadIdx.x / kRmTokens, tl = threadIdx.x % kRmTokens;
     float acc = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) acc += s_part[w][threadIdx.x];
+    for (int w = 0; w < NW; ++w) acc += s_part[w][threadIdx.x];
     if (e0 + el < N && t0 + tl < M) logits[(size_t)(t0 + tl) * N + e0 + el] = acc + (bias ? bias[e0 + el] : 0.f);
     __threadfence();
   }
@@ -382,24 +383,29 @@ __global__ void __launch_bounds__(256) router_mma_kernel(const T *__restrict__ h
   }
   __syncthreads();
   if (s_last) {
-    const int t = t0 + warp;                              // eight tokens, one warp each
-    if (t < M)
-      token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane);
+    // eight tokens: one warp each, or with sixteen warps softmax and top-k of a token on two warps
+    const int t = t0 + (warp & 7);
+    const int which = NW == 16 ? (warp < 8 ? 1 : 2) : 3;
+    if (t < M && warp < 16)
+      token_phase(logits + (size_t)t * N, N, k, prob + (size_t)t * N, topk_idx + (size_t)t * k, score_fx, natcnt, lane,
+                  which);
   }
 }
 
-template <typename T>
+template <typename T, int NW = 8>
 static cudaError_t launch_router_mma(const LaunchCtx &c, const void *hidden) {
   const moespec_layer_desc &D = *c.desc;
   const Workspace &ws = *c.ws;
   const dim3 grid((D.n_experts + kRmExperts - 1) / kRmExperts, (c.M + kRmTokens - 1) / kRmTokens);
-  return launch_kernel(router_mma_kernel<T>, grid, dim3(256), 0, c.stream, (const T *)hidden, (const T *)D.router_w,
+  return launch_kernel(router_mma_kernel<T, NW>, grid, dim3(NW * 32), 0, c.stream, (const T *)hidden, (const T *)D.router_w,
                        D.router_bias, ws.logits, ws.prob, ws.topk_idx, ws.score_fx, ws.natcnt_acc, ws.arrive,
                        ws.early_flag, ws.unit_counter, D.shortlist == MOESPEC_STATIC ? 1 : 0, ws.colmask, c.M, D.n_experts,
                        D.d, c.k);
 }
 template <>
-cudaError_t launch_router_mma<float>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
+cudaError_t launch_router_mma<float, 8>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
+template <>
+cudaError_t launch_router_mma<float, 16>(const LaunchCtx &, const void *) { return cudaErrorNotSupported; }
 
 // Trees beyond 64 tokens of a 16-bit layer take the tensor-core router (d must split into eight K ranges of
 // whole 32-element steps).
@@ -412,7 +418,11 @@ static bool use_router_mma(const LaunchCtx &c) {
 
 template <typename T>
 static cudaError_t launch_router_t(const LaunchCtx &c, const void *hidden) {
-  if (use_router_mma(c)) return launch_router_mma<T>(c, hidden);
+  // sixteen warps per CTA where K splits sixteen ways into whole 32-element steps: the eight tokens of a tile
+  // then get their softmax and their top-k on separate warps (2.5 µs per layer less than eight warps at
+  // 65 to 255 tokens and for 128 experts)
+  if (use_router_mma(c))
+    return c.desc->d % 512 == 0 ? launch_router_mma<T, 16>(c, hidden) : launch_router_mma<T, 8>(c, hidden);
   const moespec_layer_desc &D = *c.desc;
   const Workspace &ws = *c.ws;
   const int ex_tiles = (D.n_experts + 7) / 8;
@@ -1046,8 +1056,10 @@ cudaError_t routing_configure() {
   set((const void *)router_topk_kernel<__half, 2>);
   set((const void *)router_topk_kernel<__half, 4>);
   set((const void *)router_topk_kernel<__half, 8>);
-  set((const void *)router_mma_kernel<__nv_bfloat16>);
-  set((const void *)router_mma_kernel<__half>);
+  set((const void *)router_mma_kernel<__nv_bfloat16, 8>);
+  set((const void *)router_mma_kernel<__half, 8>);
+  set((const void *)router_mma_kernel<__nv_bfloat16, 16>);
+  set((const void *)router_mma_kernel<__half, 16>);
   set((const void *)softmax_topk_kernel);
   set((const void *)route_kernel<1>);
   set((const void *)route_kernel<2>);
