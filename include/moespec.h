@@ -237,7 +237,8 @@ int moespec_get_logits(moespec_layer_t *layer, float *logits_host);
 
 /* Copy an intermediate of the last verify call to a HOST buffer of `bytes` bytes
  * (clipped to the buffer's size in the workspace).  which: 0 = gathered rows
- * x_perm [R, d] in dtype (Appendix C gather), 1 = h_mid [R, f] in dtype
+ * x_perm [R, d] in dtype (Appendix C gather; not made by the tensor-core path for
+ * trees of at most 16 tokens), 1 = h_mid [R, f] in dtype
  * (silu(W1 x) * (W3 x) of the expert FFN), 2 = y [R, d] fp32 (expert outputs
  * before the gate-weighted sum).  Rows follow perm_row2tok.  Synchronises. */
 int moespec_get_intermediate(moespec_layer_t *layer, int which, void *host_buf, long long bytes);
@@ -261,7 +262,8 @@ int moespec_debug_set_wait(moespec_layer_t *layer, long long limit_cycles, int r
  * last verify call and writes the duration in milliseconds of each of its
  * kernels, in launch order, into ms[0 .. min(capacity, *n_kernels)).  bf16 tensor-core
  * layers launch four kernels (router + softmax + top-k; routing; gather; expert FFN +
- * combine); CUDA-core layers launch six (router, routing, gather, FFN gate/up, FFN
+ * combine), three for trees of at most 16 tokens (no gather: every gate/up unit then
+ * takes all tokens straight from hidden); CUDA-core layers launch six (router, routing, gather, FFN gate/up, FFN
  * down, combine). */
 int moespec_set_profiling(moespec_layer_t *layer, int on);
 int moespec_get_kernel_times(moespec_layer_t *layer, float *ms, int capacity, int *n_kernels);

@@ -253,6 +253,7 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   if (L->use_tc) {
     c.ru = tc_rows_per_unit(L->desc, M, k, c.B);
     c.early = tc_early_start(*desc, M) ? 1 : 0;
+    c.dense_all = tc_dense_all(*desc, M) ? 1 : 0;
     // The early units follow the shortlist's rank order.  Router-based ranks follow the tokens' own
     // probabilities, so the leading experts have rows; a fixed ordering (Eq. 4) does not look at the tree,
     // and with few tokens most of its leading experts get none: the early units would stream unused weights.
@@ -274,8 +275,10 @@ int run_layer(moespec_layer *L, const void *hidden, int M, int k, int B, void *o
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
   if ((e = launch_route_after_router(c)) != cudaSuccess) return cuda_fail(e);
   if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
-  if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
-  if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  if (!c.dense_all) {      // (trees of at most 16 tokens need no gathered rows on the tensor-core path)
+    if ((e = launch_gather(c, hidden)) != cudaSuccess) return cuda_fail(e);
+    if ((e = mark(++launches)) != cudaSuccess) return cuda_fail(e);
+  }
   if (L->use_tc) {
     // both FFN phases and the combine are one persistent kernel
     if ((e = launch_ffn_tensor_core(c, &L->maps, hidden, out)) != cudaSuccess) return cuda_fail(e);

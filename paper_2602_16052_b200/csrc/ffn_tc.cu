@@ -323,6 +323,16 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     sentinel.expert = -1; sentinel.tile = 0; sentinel.row0 = 0; sentinel.n_rows = 0; sentinel.chunk = 0;
     sentinel.phase = 0; sentinel.pad0 = 0; sentinel.pad1 = 0;
     Unit un = sentinel;
+    // A list entry marked 2 is a gate/up unit of a tree so small that every unit takes all tokens from `hidden`
+    // (no gathered copy exists): it runs like an early unit, and its epilogue finds its rows in the entry.
+    auto from_list = [&](int u) -> Unit {
+      Unit x = a.units[u];
+      if (x.pad0 == 2) {
+        if (x.n_rows == 0) x.pad0 = 0;             // no rows: skipped like any other empty unit
+        else { x.pad0 = 1; x.pad1 = u; x.n_rows = a.M; x.row0 = 0; }
+      }
+      return x;
+    };
     // the first ticket (the router kernel of this call left the dispenser at zero)
     int t_first = 0;
     if (lane == 0) t_first = atomicAdd(a.unit_counter, 1);
@@ -360,7 +370,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     }
     if (waited) {
       n_total = a.n_units[0] + a.n_units[1];
-      if (lane == 0 && !un.pad0 && t_first < n_total) un = a.units[t_first];
+      if (lane == 0 && !un.pad0 && t_first < n_total) un = from_list(t_first);
     }
     while (ok) {
       Unit un_next = sentinel;
@@ -371,7 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         while (un.expert >= 0 && un.n_rows == 0 && !un.pad0) {
           if (un.phase == 1) atomicAdd(a.down_done, 1);
           const int u2 = atomicAdd(a.unit_counter, 1);
-          un = u2 < n_total ? a.units[u2] : sentinel;
+          un = u2 < n_total ? from_list(u2) : sentinel;
         }
         const uint32_t q = qi % kQueue, qph = (qi / kQueue) & 1u;
         if (!mbar_wait(bar_q_empty + 8 * q, qph ^ 1u, abort_flag, a.spin_limit)) ok = 0;
@@ -489,7 +499,7 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       }
       it += (uint32_t)armed;                        // == k_iters unless the CTA is aborting
       if (!ok) break;
-      if (lane == 0 && u_next < n_total) un_next = a.units[u_next];
+      if (lane == 0 && u_next < n_total) un_next = from_list(u_next);
       un = un_next;
     }
     if (!ok && lane == 0) {
@@ -859,6 +869,8 @@ cudaError_t tc_configure() {
 }
 
 // Early start needs every token in one MMA (N <= 128) and is an option of the tensor-core path.
+bool tc_dense_all(const moespec_layer_desc &d, int M) { return is_16bit(d.dtype) && M >= 1 && M <= kTokBoxSmall; }
+
 bool tc_early_start(const moespec_layer_desc &d, int M) {
   static const bool off = [] { const char *v = experiment_env("MOESPEC_NO_EARLY"); return v && v[0] == '1'; }();
   return !off && is_16bit(d.dtype) && M >= 1 && M <= kMaxTokChunk;
@@ -943,7 +955,7 @@ cudaError_t launch_ffn_tensor_core(const LaunchCtx &c, const TcMaps *maps, const
   a.static_order = c.ws->static_order;
   if (a.early && D.shortlist == MOESPEC_STATIC) a.static_nS = c.B < c.ws->n_static ? c.B : c.ws->n_static;
   TcMapsCall m;
-  if (a.early) {
+  if (a.early || c.dense_all) {
     // the call's input as a TMA tensor [M, d]: rows beyond M read as zeros
     if (maps->hidden_ptr != hidden || maps->hidden_M != c.M) {
       EncodeTiledFn enc = nullptr;

@@ -96,6 +96,8 @@ struct LaunchCtx {
   cudaStream_t stream;
   int ru;               // weight rows per tensor-core work unit for this call (0: CUDA-core path)
   int early = 0;        // 1: the FFN kernel starts on the shortlist before routing has finished (see ffn_tc.cu)
+  int dense_all = 0;    // 1: every gate/up unit takes ALL tokens straight from `hidden` (trees of at most 16
+                        //    tokens: the smallest MMA holds them anyway), so no gathered copy is made
   int res_first = 0, res_count = 0; // resident experts [res_first, res_first + res_count) (res_count = N: all)
   long long debug_spin_limit = 0;   // test hook: bound of device-side waits in cycles (0 = default)
   int debug_ready_bias = 0;         // test hook: extra slabs every down unit waits for (never reported)
@@ -160,6 +162,7 @@ int tc_rows_per_unit(const moespec_layer_desc &d, int M, int k, int B);   // gat
 int tc_rows_per_down_unit(int ru);                                         // down slab height for a call
 int tc_grid_size(int device);                                              // CTAs of the FFN kernel (one per SM)
 bool tc_early_start(const moespec_layer_desc &d, int M);                  // does a call of M tokens use early start?
+bool tc_dense_all(const moespec_layer_desc &d, int M);                    // ... and no gathered rows at all?
 cudaError_t tc_encode_maps(const moespec_layer_desc &d, const Workspace &ws, int R_cap, TcMaps *maps,
                            int *cu_result);
 cudaError_t tc_configure();   // one-time function attributes

@@ -494,6 +494,7 @@ struct RouteArgs {
   int ffn_ctas;                 // CTAs of the FFN kernel: CTA c starts on gate/up unit c of the list
   int rows_later;               // the row of every (token, slot) pair is left to the row kernel (large trees)
   int res_first, res_count;     // experts resident on this GPU (expert-parallel shard); res_count = N: all
+  int dense_all;                // gate/up units are marked "all tokens from hidden" (trees of at most 16 tokens)
 };
 
 constexpr int kRouteWarps = 8;      // tokens per CTA of route_kernel
@@ -850,7 +851,8 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         const int cpos = v / tiles;           // position in chunk-prefix space: identifies the expert
         if (a.early) {                        // one chunk per listed expert, rank order
           const int e1 = s_chunk_expert[cpos];
-          ws.units[u] = Unit{e1, v - cpos * tiles, s_offset[e1], s_count[e1], cpos, phase, 0, 0};
+          ws.units[u] = Unit{e1, v - cpos * tiles, s_offset[e1], s_count[e1], cpos, phase,
+                             (a.dense_all && !phase) ? 2 : 0, 0};
           continue;
         }
         int e;
@@ -867,7 +869,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         const int tl = local / chunks_e, c = local - tl * chunks_e;
         const int row0 = s_offset[e] + c * kMaxTokChunk;
         const int rows = min(kMaxTokChunk, s_count[e] - c * kMaxTokChunk);
-        ws.units[u] = Unit{e, tl, row0, rows, s_unit_base[e] + c, phase, 0, 0};
+        ws.units[u] = Unit{e, tl, row0, rows, s_unit_base[e] + c, phase, (a.dense_all && !phase) ? 2 : 0, 0};
       }
     }
   } else if (warp == 7) {
@@ -922,6 +924,7 @@ static cudaError_t launch_route_kernel(const LaunchCtx &c, const float *logits) 
   a.early = c.ru > 0 ? c.early : 0;
   a.ffn_ctas = tc_grid_size(D.device);
   a.rows_later = rows_in_row_kernel(c.M);
+  a.dense_all = c.ru > 0 ? c.dense_all : 0;
   a.res_first = c.res_count > 0 ? c.res_first : 0;
   a.res_count = c.res_count > 0 ? c.res_count : D.n_experts;
   const dim3 grid((c.M + kRouteWarps - 1) / kRouteWarps), block(kRouteWarps * 32);

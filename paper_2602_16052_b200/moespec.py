@@ -290,6 +290,7 @@ class Layer:
         return st.as_dict()
 
     KERNEL_NAMES_TC = ("router_topk", "route", "gather", "ffn")
+    KERNEL_NAMES_TC_SMALL = ("router_topk", "route", "ffn")      # trees of at most 16 tokens: no gathered copy
     KERNEL_NAMES_CC = ("router_topk", "route", "gather", "ffn_gate_up", "ffn_down", "combine")
 
     def debug_set_wait(self, limit_cycles: int, ready_bias: int):
@@ -305,7 +306,7 @@ class Layer:
         n = C.c_int(0)
         _check(lib().moespec_get_kernel_times(self._h, C.cast(ms, C.c_void_p), 8, C.cast(C.byref(n), C.c_void_p)),
                "moespec_get_kernel_times")
-        names = self.KERNEL_NAMES_TC if n.value == len(self.KERNEL_NAMES_TC) else self.KERNEL_NAMES_CC
+        names = {3: self.KERNEL_NAMES_TC_SMALL, 4: self.KERNEL_NAMES_TC}.get(n.value, self.KERNEL_NAMES_CC)
         return {names[i]: float(ms[i]) for i in range(min(n.value, len(names)))}
 
     def last_launch_count(self) -> int:
