@@ -998,6 +998,15 @@ __global__ void __launch_bounds__(128) rows_gather_kernel(const uint4 *__restric
   const int lane = threadIdx.x & 31;
   __shared__ int s_row;
   pdl_trigger();
+  // The token's hidden state does not depend on the routing (it is the layer's input, valid since the router
+  // kernel's wait): its first 8 KB are on their way before this kernel waits for the routing kernel, so the
+  // chain behind that wait is "expert of the slot -> bit-matrix row and offset -> stores" only.
+  constexpr int PRE = 4;
+  const uint4 *src = hidden ? hidden + (size_t)t * row_vec : nullptr;
+  uint4 pre[PRE];
+#pragma unroll
+  for (int u = 0; u < PRE; ++u)
+    if (hidden && (int)threadIdx.x + u * 128 < row_vec) pre[u] = src[threadIdx.x + u * 128];
   pdl_wait();
   const int e = assign_idx[pair];
   if (e < 0) {                                  // dropped slot (truncation, or fewer than k experts kept)
@@ -1007,13 +1016,14 @@ __global__ void __launch_bounds__(128) rows_gather_kernel(const uint4 *__restric
   if (threadIdx.x < 32) {
     const unsigned *cm = colmask + (size_t)e * ((M + 31) >> 5);
     const int full = t >> 5;
+    const int off = lane == 0 ? offset[e] : 0;          // in flight together with the bit-matrix words
     int below = 0;
     for (int w = lane; w < full; w += 32) below += __popc(cm[w]);
     if (lane == 0) below += __popc(cm[full] & ((1u << (t & 31)) - 1u));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(kFull, below, o);
     if (lane == 0) {
-      const int row = offset[e] + below;
+      const int row = off + below;
       s_row = row;
       perm_row2tok[row] = t;
       if (row2expert) row2expert[row] = e;
@@ -1022,9 +1032,11 @@ __global__ void __launch_bounds__(128) rows_gather_kernel(const uint4 *__restric
   }
   if (!hidden) return;
   __syncthreads();
-  const uint4 *src = hidden + (size_t)t * row_vec;
   uint4 *dst = x_perm + (size_t)s_row * row_vec;
-  for (int j = threadIdx.x; j < row_vec; j += blockDim.x) dst[j] = src[j];
+#pragma unroll
+  for (int u = 0; u < PRE; ++u)
+    if ((int)threadIdx.x + u * 128 < row_vec) dst[threadIdx.x + u * 128] = pre[u];
+  for (int j = threadIdx.x + PRE * 128; j < row_vec; j += blockDim.x) dst[j] = src[j];
 }
 
 cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
