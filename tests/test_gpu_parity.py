@@ -350,6 +350,26 @@ def test_residual_and_host_entry_point():
     layer.destroy()
 
 
+def test_host_entry_alternating_between_trees_and_buffers():
+    """The host entry point keeps a few captured graphs: a caller that alternates between two trees and two
+    buffer pairs must get, on every call, the result of the device entry point for that call's arguments."""
+    cfg = synth.CONFIGS["olmoe"].with_(f=128)
+    case = H.make_case(cfg, 63, seed=16)
+    layer = make_layer(case, 63, 8)
+    variants = []
+    for M, B in ((63, 32), (40, 12), (17, 8)):
+        h_dev = case["hidden"][:M].contiguous()
+        variants.append((M, B, h_dev.cpu().pin_memory(), torch.empty((M, cfg.d), dtype=h_dev.dtype).pin_memory(),
+                         layer.verify_layer(h_dev, 8, B).cpu()))
+    torch.cuda.synchronize()
+    for rnd in range(3):
+        for M, B, h_host, o_host, want in variants:
+            o_host.zero_()
+            layer.verify_layer_host(h_host, 8, B, o_host)
+            assert torch.equal(o_host, want), (rnd, M, B)
+    layer.destroy()
+
+
 def test_repeat_calls_are_bitwise_reproducible():
     cfg = synth.CONFIGS["olmoe"].with_(f=256)
     case = H.make_case(cfg, 127, seed=8)
