@@ -556,14 +556,15 @@ def run_reference(args):
         return
     cfg = synth.CONFIGS[WORKLOAD]
     case = oracle_case(cfg, M_TOKENS, seed=1000)
-    for _ in range(min(args.warmup, 1)):
+    warm = min(args.warmup, 3)
+    for _ in range(warm):
         time_oracle(cfg, M_TOKENS, B_HEADLINE, 0.0, 1, case)
-    steps = max(1, min(args.steps, 5))
+    steps = max(1, min(args.steps, 200))       # a layer takes ~50 ms on the host cores: K steps as asked, up to ~10 s
     us, cores, reps = time_oracle(cfg, M_TOKENS, B_HEADLINE, 1e9, steps, case)
     sample = f"{reps} whole verify layers (M={M_TOKENS}, B={B_HEADLINE}) of the same workload, median"
     line = {
         "impl": "reference", "metric": METRIC, "value": us, "unit": "us", "n_gpus": args.gpus, "steps": reps,
-        "warmup": min(args.warmup, 1), "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
+        "warmup": warm, "ms_per_step": us / 1e3, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": workload_name(cfg)},
         "cpu_baseline": {"value": us, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample},
