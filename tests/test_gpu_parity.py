@@ -357,7 +357,7 @@ def test_host_entry_alternating_between_trees_and_buffers():
     case = H.make_case(cfg, 63, seed=16)
     layer = make_layer(case, 63, 8)
     variants = []
-    for M, B in ((63, 32), (40, 12), (17, 8)):
+    for M, B in ((63, 32), (40, 12), (17, 8), (7, 16)):      # (7 tokens: the path without a gathered copy)
         h_dev = case["hidden"][:M].contiguous()
         variants.append((M, B, h_dev.cpu().pin_memory(), torch.empty((M, cfg.d), dtype=h_dev.dtype).pin_memory(),
                          layer.verify_layer(h_dev, 8, B).cpu()))
