@@ -250,6 +250,11 @@ __device__ __forceinline__ int ld_acquire(const int *p) {
   asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// Release increment by one thread after a CTA barrier: the stores of all threads that arrived at the barrier are
+// visible to whoever acquires the new value.
+__device__ __forceinline__ void red_release_add(int *p) {
+  asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p) : "memory");
+}
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void epilogue_bar() { asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory"); }
 
@@ -275,6 +280,14 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_stages = a.n_stages;
   pdl_trigger();
+  // The first ticket and, with early start, the first 32 shortlist words are requested before anything else:
+  // their round trips through L2 overlap the set-up below.  (The router kernel of this call left the
+  // dispenser at zero and has completed, or with a fixed shortlist has at least performed that reset.)
+  int t_first = 0, w_pre = 0;
+  if (warp == 0) {
+    if (lane == 0) t_first = atomicAdd(a.unit_counter, 1);
+    if (a.early && a.static_nS == 0 && lane < a.n_words) w_pre = ld_acquire(a.early_flag + lane);
+  }
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < n_stages; ++s) {
@@ -333,23 +346,23 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       }
       return x;
     };
-    // the first ticket (the router kernel of this call left the dispenser at zero)
-    int t_first = 0;
-    if (lane == 0) t_first = atomicAdd(a.unit_counter, 1);
     if (a.early) {
       // The routing kernel publishes the shortlist long before the gather order exists.  Ticket c below the
       // grid size is gate/up unit c of the rank-ordered list (expert S_rank[c / tiles], slab c % tiles) and
       // is started on with ALL tokens as the MMA's N dimension, read straight from `hidden`; the epilogue
       // keeps the routed tokens only.  The routing kernel builds the unit list in the same order and keeps
       // the experts of those ranks in it even without rows, so unit c of the list is this unit.
+      const int r_first = __shfl_sync(0xffffffffu, t_first, 0) / a.tiles_real;
+      const int v_pre = __shfl_sync(0xffffffffu, w_pre, r_first & 31);      // that rank's word as read at entry
       if (lane == 0 && t_first < (int)gridDim.x) {
-        const int r = t_first / a.tiles_real;
+        const int r = r_first;
         int v = -1;                      // the expert of rank r, plus one
         if (a.static_nS > 0) {           // a fixed shortlist needs no publication: stream from the first cycle
           if (r < a.static_nS) v = a.static_order[r] + 1;
         } else if (r < a.n_words) {
           const long long t0 = clock64();
-          while ((v = ld_acquire(a.early_flag + r)) == 0) {
+          v = r < 32 ? v_pre : 0;
+          while (v == 0 && (v = ld_acquire(a.early_flag + r)) == 0) {
             if (*abort_flag || clock64() - t0 > a.spin_limit) { *abort_flag = 1; ok = 0; break; }
             __nanosleep(32);
           }
@@ -627,10 +640,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
         }
         tc_fence_before();
         mbar_arrive(bar_acc_empty + 8 * ab);
-        __threadfence();
         fence_proxy_async();
         epilogue_bar();
-        if (threadIdx.x == 64) atomicAdd(a.ready + real.chunk, 1);
+        if (threadIdx.x == 64) red_release_add(a.ready + real.chunk);
         mbar_arrive(bar_q_empty + 8 * q);
         ++acc_it;
         continue;
@@ -682,10 +694,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
       mbar_arrive(bar_acc_empty + 8 * ab);
       // publish the slab (h_mid for a gate/up unit, y for a down unit): every thread's stores are
       // fenced, then one thread bumps the counter the consumers of the slab watch
-      __threadfence();
       if (un.phase == 0) fence_proxy_async();
       epilogue_bar();
-      if (threadIdx.x == 64) atomicAdd(un.phase == 0 ? a.ready + un.chunk : a.down_done, 1);
+      if (threadIdx.x == 64) red_release_add(un.phase == 0 ? a.ready + un.chunk : a.down_done);
       mbar_arrive(bar_q_empty + 8 * q);
       ++acc_it;
     }

@@ -42,6 +42,14 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Arrival at a counter by one thread after a CTA barrier: releases the stores of every thread of the CTA that
+// came before the barrier, and acquires those released by the CTAs that arrived earlier.
+__device__ __forceinline__ int arrive_acq_rel(int *counter) {
+  int prev;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], 1;" : "=r"(prev) : "l"(counter) : "memory");
+  return prev;
+}
+
 // ---------------------------------------------------------------------------
 // Warp-wide ranking under (value descending, expert index ascending).  Lane l
 // owns experts l, l+32, ...; `valid` has bit s set while local slot s is still
@@ -255,16 +263,12 @@ __global__ void __launch_bounds__(256) router_topk_kernel(const T *__restrict__ 
       for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(kFull, a, o);
       if (lane == 0 && t0 + tt < M) logits[(size_t)(t0 + tt) * N + i] = a + b;
     }
-    if (lane == 0) __threadfence();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int prev = atomicAdd(&arrive[blockIdx.y], 1);
+    const int prev = arrive_acq_rel(&arrive[blockIdx.y]);
     s_last = (prev == (int)gridDim.x - 1);
-    if (s_last) {
-      arrive[blockIdx.y] = 0;
-      __threadfence();
-    }
+    if (s_last) arrive[blockIdx.y] = 0;
   }
   __syncthreads();
   if (s_last) {
@@ -370,16 +374,12 @@ __global__ void __launch_bounds__(NW * 32) router_mma_kernel(const T *__restrict
 #pragma unroll
     for (int w = 0; w < NW; ++w) acc += s_part[w][threadIdx.x];
     if (e0 + el < N && t0 + tl < M) logits[(size_t)(t0 + tl) * N + e0 + el] = acc + (bias ? bias[e0 + el] : 0.f);
-    __threadfence();
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    const int prev = atomicAdd(&arrive[blockIdx.y], 1);
+    const int prev = arrive_acq_rel(&arrive[blockIdx.y]);
     s_last = (prev == (int)gridDim.x - 1);
-    if (s_last) {
-      arrive[blockIdx.y] = 0;
-      __threadfence();
-    }
+    if (s_last) arrive[blockIdx.y] = 0;
   }
   __syncthreads();
   if (s_last) {
@@ -716,12 +716,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   if (t < M) route_token<W>(a, t, nS, s_Smask, key, p, nat, lane);
 
   // ---- the CTA that arrives last finishes the call
-  __threadfence();
   __syncthreads();
   if (tid == 0) {
-    const int prev = atomicAdd(ws.arrive_route, 1);
+    const int prev = arrive_acq_rel(ws.arrive_route);
     s_last = (prev == (int)gridDim.x - 1);
-    if (s_last) __threadfence();
   }
   __syncthreads();
   if (!s_last) return;
