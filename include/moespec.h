@@ -237,8 +237,10 @@ int moespec_get_logits(moespec_layer_t *layer, float *logits_host);
 
 /* Copy an intermediate of the last verify call to a HOST buffer of `bytes` bytes
  * (clipped to the buffer's size in the workspace).  which: 0 = gathered rows
- * x_perm [R, d] in dtype (Appendix C gather; not made by the tensor-core path for
- * trees of at most 16 tokens), 1 = h_mid [R, f] in dtype
+ * x_perm [R, d] in dtype (Appendix C gather; on the tensor-core path not made for
+ * trees of at most 16 tokens, and for trees of at most 128 tokens made only for
+ * the experts some of whose gate/up work reads it: the best-ranked experts'
+ * rows are taken straight from hidden), 1 = h_mid [R, f] in dtype
  * (silu(W1 x) * (W3 x) of the expert FFN), 2 = y [R, d] fp32 (expert outputs
  * before the gate-weighted sum).  Rows follow perm_row2tok.  Synchronises. */
 int moespec_get_intermediate(moespec_layer_t *layer, int which, void *host_buf, long long bytes);

@@ -170,6 +170,7 @@ size_t carve(const moespec_layer_desc &d, int R_cap, char *base, Workspace *ws) 
   c.take(w.offset, N + 1);
   c.take(w.active, N);
   c.take(w.perm_row2tok, (size_t)R_cap);
+  c.take(w.gather_src, (size_t)R_cap);
   c.take(w.row2expert, (size_t)R_cap);
   c.take(w.tokslot2row, M * K);
   w.mask_words = (int)((M + 31) / 32);

@@ -336,8 +336,9 @@ __global__ void __launch_bounds__(kThreads, 1) ffn_tc_kernel(const __grid_consta
     sentinel.expert = -1; sentinel.tile = 0; sentinel.row0 = 0; sentinel.n_rows = 0; sentinel.chunk = 0;
     sentinel.phase = 0; sentinel.pad0 = 0; sentinel.pad1 = 0;
     Unit un = sentinel;
-    // A list entry marked 2 is a gate/up unit of a tree so small that every unit takes all tokens from `hidden`
-    // (no gathered copy exists): it runs like an early unit, and its epilogue finds its rows in the entry.
+    // A list entry marked 2 is a gate/up unit that takes all tokens from `hidden`: one of the first units of the
+    // list, which CTAs may have started on early, or any unit of a tree so small that no gathered copy is made.
+    // It runs like an early unit, and its epilogue finds its rows in the entry.
     auto from_list = [&](int u) -> Unit {
       Unit x = a.units[u];
       if (x.pad0 == 2) {

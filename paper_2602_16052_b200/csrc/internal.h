@@ -58,6 +58,8 @@ struct Workspace {
   int *offset;          // [N+1]
   int *active;          // [N]
   int *perm_row2tok;    // [R_cap]
+  int *gather_src;      // [R_cap] token whose hidden state row r of x_perm is a copy of, or -1 when no work unit
+                        // reads that row (every gate/up unit of its expert takes all tokens from hidden); may be null
   int *row2expert;      // [R_cap]
   int *tokslot2row;     // [max_M, max_k]
   // accumulators shared by the CTAs of one call; every one of them is zero between calls (the routing

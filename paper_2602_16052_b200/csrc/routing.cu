@@ -598,6 +598,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   __shared__ unsigned long long s_warp_tot[kRouteWarps];
   __shared__ int s_chunk_expert[kMaxExperts * 2];     // token chunk -> expert (first 2N chunks; more fall back)
   __shared__ int s_nactive, s_last, s_nchunks;
+  __shared__ unsigned char s_all_dense[kMaxExperts];   // expert whose gate/up units all take every token from hidden
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int M = a.M, N = a.N, k = a.k;
@@ -723,6 +724,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
   }
   __syncthreads();
   if (!s_last) return;
+  if (tid < N) s_all_dense[tid] = 0;      // (set below, behind a barrier, for trees with early start)
 
   // rows per expert and exclusive scans of rows, token chunks and active experts (Appendix C gather)
   const int used_words = (M + 31) >> 5;
@@ -770,12 +772,16 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     // Early start (M <= 128, so an expert has at most one token chunk): the unit list follows the
     // shortlist's rank order, and the experts whose gate/up units the FFN kernel's CTAs start on before
     // this list exists (CTA c takes unit c) keep their place even if no token was routed to them.
+    // The gate/up units that CTAs may start on early (the first `ffn_ctas` of the list) are marked as taking
+    // all tokens from `hidden`, whoever draws them and when; an expert all of whose gate/up units are among
+    // them has no reader for its rows of the gathered copy, and they are not made.
     const int n_head = min((a.ffn_ctas + a.tiles_up - 1) / a.tiles_up, nS_l);
     bool present = false;
     int e_r = 0;
     if (tid < nS_l) {
       e_r = s_Srank[tid];
       present = s_count[e_r] > 0 || tid < n_head;
+      if ((tid + 1) * a.tiles_up <= a.ffn_ctas) s_all_dense[e_r] = 1;
     }
     const unsigned bal = __ballot_sync(kFull, present);
     if (lane == 0) s_warp_tot[warp] = (unsigned long long)__popc(bal);
@@ -831,6 +837,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
           row = s_offset[e[u]] + below;
           ws.perm_row2tok[row] = tt;
           ws.row2expert[row] = e[u];
+          if (ws.gather_src) ws.gather_src[row] = s_all_dense[e[u]] ? -1 : tt;
         }
         ws.tokslot2row[(size_t)tt * k + slot] = row;
       }
@@ -850,7 +857,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         if (a.early) {                        // one chunk per listed expert, rank order
           const int e1 = s_chunk_expert[cpos];
           ws.units[u] = Unit{e1, v - cpos * tiles, s_offset[e1], s_count[e1], cpos, phase,
-                             (a.dense_all && !phase) ? 2 : 0, 0};
+                             (!phase && (a.dense_all || u < a.ffn_ctas)) ? 2 : 0, 0};
           continue;
         }
         int e;
@@ -965,7 +972,8 @@ cudaError_t launch_route(const LaunchCtx &c, const float *logits) {
 }
 
 // ---------------------------------------------------------------------------
-// K3: gather routed rows: x_perm[r, :] = hidden[perm_row2tok[r], :] (Appendix C), one CTA per row.
+// K3: gather routed rows: x_perm[r, :] = hidden[perm_row2tok[r], :] (Appendix C), one CTA per row.  `perm` is
+// the gather order, or its copy in which the rows that no work unit reads are marked -1 and skipped.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restrict__ hidden,
                                                           uint4 *__restrict__ x_perm,
@@ -976,6 +984,7 @@ __global__ void __launch_bounds__(128) gather_rows_kernel(const uint4 *__restric
   pdl_wait();
   if (r >= counters[2]) return;
   const int t = perm[r];
+  if (t < 0) return;                       // a row that no work unit reads
   const uint4 *src = hidden + (size_t)t * row_vec;
   uint4 *dst = x_perm + (size_t)r * row_vec;
   for (int j = threadIdx.x; j < row_vec; j += blockDim.x) dst[j] = src[j];
@@ -1049,7 +1058,8 @@ cudaError_t launch_gather(const LaunchCtx &c, const void *hidden) {
                          (const unsigned *)ws.colmask, ws.perm_row2tok, ws.row2expert, ws.tokslot2row, c.M, c.k,
                          row_vec);
   return launch_kernel(gather_rows_kernel, dim3(rows), dim3(128), 0, c.stream, (const uint4 *)hidden,
-                       (uint4 *)ws.x_perm, (const int *)ws.perm_row2tok, (const int *)ws.counters, row_vec);
+                       (uint4 *)ws.x_perm, (const int *)(ws.gather_src ? ws.gather_src : ws.perm_row2tok),
+                       (const int *)ws.counters, row_vec);
 }
 
 // The FFN kernel needs nearly all of an SM's shared memory.  An SM whose L1/shared split was chosen for
