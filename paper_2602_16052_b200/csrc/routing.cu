@@ -15,8 +15,9 @@
 //                        re-routes its tokens, and the CTA that finishes last
 //                        does the scan, the gather order, the work-unit list and
 //                        the statistics
-//   gather_rows_kernel   x_perm[row] = hidden[token] (rows_gather_kernel also
-//                        works out the rows, for trees above 128 tokens)
+//   gather_rows_kernel   x_perm[row] = hidden[token], for the rows that some work
+//                        unit reads (rows_gather_kernel also works out the rows,
+//                        for trees above 128 tokens)
 // Scores are accumulated as 2^-52 fixed-point integers, so the sum does not
 // depend on the order in which tokens arrive and identical experts tie exactly.
 // A stand-alone softmax/top-k kernel serves callers that inject logits.
