@@ -126,3 +126,25 @@ def test_shard_argument_errors():
     assert lib.moespec_layer_create(ctypes.byref(d), ctypes.byref(h)) == m.ERR_INVALID_ARG      # 13 + 4 > 16
     d.resident_first, d.resident_count = 2, 0
     assert lib.moespec_layer_create(ctypes.byref(d), ctypes.byref(h)) == m.ERR_INVALID_ARG      # a first without a count
+
+
+def test_seeded_sweep_of_sharded_layers():
+    """Sixteen seeded draws of (N, k, M, B, d, f, shortlist mode, slope, number of shards) through run_sharded:
+    uneven expert blocks (N not a multiple of the shard count), shards that end up without a kept expert,
+    trees with and without the early start."""
+    import random
+    rng = random.Random(20260218)
+    for trial in range(16):
+        N = rng.choice([4, 8, 13, 32, 64, 100])
+        k = rng.randint(1, min(N, 8))
+        M = rng.choice([1, 5, 16, 17, 63, 100, 129, 200])
+        B = rng.randint(1, N + 1)
+        cfg = synth.LayerConfig(f"epsweep{trial}", d=rng.choice([128, 256, 512]), n_experts=N, k=k,
+                                f=rng.choice([128, 256]), dtype="bf16", slope=rng.choice([0.5, 1.0, 2.0]))
+        world = rng.choice([w for w in (2, 3, 4, 8) if w <= N])
+        mode = rng.choice([orc.FROM_ALL, orc.FROM_UNION])
+        try:
+            run_sharded(cfg, M, B, world, orc.SUBSTITUTION, mode, True, ms().FFN_TENSOR_CORE, seed=400 + trial)
+        except AssertionError as e:
+            raise AssertionError(f"trial {trial}: N={N} k={k} M={M} B={B} d={cfg.d} f={cfg.f} shards={world} "
+                                 f"mode={mode}: {e}") from e

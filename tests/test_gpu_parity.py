@@ -272,6 +272,57 @@ def test_seeded_sweep_of_random_shapes_and_settings():
                                  f"mode={mode} renorm={renorm} residual={residual}: {e}") from e
 
 
+def test_seeded_sweep_of_the_other_paths():
+    """Sixty seeded draws over what the sweep above leaves out: fp32 layers on the CUDA-core kernels (1e-5
+    relative), fixed shortlists (Eq. 4) with a random ordering of random length, and 16-bit outputs with and
+    without the residual."""
+    import random
+    rng = random.Random(20260217)
+    for trial in range(60):
+        kind = ("fp32", "static", "out16")[trial % 3]
+        N = rng.choice([4, 8, 13, 32, 64, 100, 128])
+        k = rng.randint(1, min(N, 8))
+        M = rng.choice([1, 5, 16, 17, 33, 63, 64, 100, 128, 129, 200])
+        B = rng.randint(1, N + 1)
+        d = rng.choice([128, 256, 512])
+        f = rng.choice([128, 256, 384])
+        policy = rng.choice([orc.SUBSTITUTION, orc.SUBSTITUTION, orc.TRUNCATION])
+        mode = rng.choice([orc.FROM_ALL, orc.FROM_UNION])
+        renorm = rng.random() < 0.7
+        slope = rng.choice([0.5, 1.0, 2.0])
+        residual = rng.random() < 0.4
+        try:
+            if kind == "fp32":
+                cfg = synth.LayerConfig(f"other{trial}", d=d, n_experts=N, k=k, f=f, dtype="fp32", slope=slope)
+                run_e2e(cfg, M, B, policy, mode, renorm, ms().FFN_CUDA_CORE, seed=300 + trial, residual=residual)
+            elif kind == "out16":
+                dt = rng.choice(["bf16", "fp16"])
+                cfg = synth.LayerConfig(f"other{trial}", d=d, n_experts=N, k=k, f=f, dtype=dt, slope=slope)
+                run_e2e(cfg, M, B, orc.SUBSTITUTION, mode, True, ms().FFN_TENSOR_CORE, seed=300 + trial, residual=residual,
+                        out_dtype=torch.bfloat16 if dt == "bf16" else torch.float16)
+            else:
+                cfg = synth.LayerConfig(f"other{trial}", d=d, n_experts=N, k=k, f=f, dtype="bf16", slope=slope)
+                case = H.make_case(cfg, M, 300 + trial)
+                order = list(range(N))
+                rng.shuffle(order)
+                order = order[:rng.randint(1, N)]
+                layer = make_layer(case, M, k, shortlist=ms().STATIC, out_dtype=torch.float32)
+                layer.set_static_ranking(order)
+                out = layer.verify_layer(case["hidden"], k, B)
+                torch.cuda.synchronize()
+                assert layer.get_stats()["status"] == 0
+                r = orc.verify_layer(H.f64(case["hidden"]), H.f64(case["router_w"]), H.f64(case["router_bias"]),
+                                     H.LazyF64(case["w_gate"]), H.LazyF64(case["w_up"]), H.LazyF64(case["w_down"]), k, B,
+                                     orc.SUBSTITUTION, orc.STATIC, True, logits=layer.get_logits(), static_rank=order)
+                assert r["S"] == order[:B]
+                H.compare_routing(layer.get_routing(), r, orc.SUBSTITUTION, k)
+                check_out(out, r["out"], "bf16")
+                layer.destroy()
+        except AssertionError as e:
+            raise AssertionError(f"trial {trial} ({kind}): N={N} k={k} M={M} B={B} d={d} f={f} policy={policy} "
+                                 f"mode={mode} renorm={renorm} residual={residual} slope={slope}: {e}") from e
+
+
 def test_error_beyond_the_bar_is_the_16_bit_intermediate():
     """Truncation with raw gating on flat routing gives rows whose norms differ several-fold, and max |err|
     against the all-rows RMS then exceeds 2e-2 on a few random shapes (six of 876 draws of a longer soak, at
