@@ -799,11 +799,42 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       s_nchunks = tot;
     }
     __syncthreads();
+  } else if (a.tiles_up > 0) {
+    // Larger trees: the listed experts in the shortlist's rank order too, each with its token chunks.  Rank
+    // order is roughly row-count order, so the units that take longest (two or more full chunks, whose slabs
+    // are re-read by every chunk) are handed out first and the list ends with the cheap ones; in expert-index
+    // order whatever expert came last decided how long the CTAs waited for the last of them.
+    int e_r = 0, ch = 0;
+    if (tid < nS_l) {
+      e_r = s_Srank[tid];
+      ch = (s_count[e_r] + kMaxTokChunk - 1) / kMaxTokChunk;
+    }
+    int inc = ch;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int up = __shfl_up_sync(kFull, inc, o);
+      if (lane >= o) inc += up;
+    }
+    if (lane == 31) s_warp_tot[warp] = (unsigned long long)inc;
+    __syncthreads();                       // (also: every thread is done with the index-order bases)
+    int pre = inc - ch;
+    for (int w = 0; w < warp; ++w) pre += (int)s_warp_tot[w];
+    if (tid < nS_l) {
+      s_unit_base[e_r] = pre;
+      s_cand[e_r] = ch;                    // (the candidate flags are no longer needed: chunk count per expert)
+      for (int cc = 0; cc < ch && pre + cc < 2 * kMaxExperts; ++cc) s_chunk_expert[pre + cc] = e_r;
+    }
+    if (tid == 0) {
+      int tot = 0;
+      for (int w = 0; w < kRouteWarps; ++w) tot += (int)s_warp_tot[w];
+      s_nchunks = tot;
+    }
+    __syncthreads();
   }
 
   // The rest is three independent jobs, each latency-bound, run side by side:
   //   warps 0-3  row of every (token, slot)       warps 4-6  work-unit list       warp 7  coverage
-  const int n_chunks = a.early ? s_nchunks : s_unit_base[N];
+  const int n_chunks = a.tiles_up > 0 ? s_nchunks : s_unit_base[N];
   double cov = 0.0;
   if (warp < 4 && !a.rows_later) {
     // rows ordered by (expert ascending, token ascending): the row of (t, e) is
@@ -864,13 +895,14 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         int e;
         if (cpos < 2 * kMaxExperts) {
           e = s_chunk_expert[cpos];
-        } else {          // more than 2N token chunks (M far beyond 128): search the chunk bases
-          e = 0;
-          while (s_unit_base[e + 1] <= cpos) ++e;
+        } else {          // more than 2N token chunks (M far beyond 128): search the chunk bases, in rank order
+          int r = 0;
+          e = s_Srank[0];
+          while (s_unit_base[e] + s_cand[e] <= cpos) e = s_Srank[++r];
         }
         // inside an expert: slab-major, token chunk innermost, so the chunks that re-read a slab are
         // handed out back to back and the second read hits L2
-        const int chunks_e = s_unit_base[e + 1] - s_unit_base[e];
+        const int chunks_e = s_cand[e];
         const int local = v - s_unit_base[e] * tiles;
         const int tl = local / chunks_e, c = local - tl * chunks_e;
         const int row0 = s_offset[e] + c * kMaxTokChunk;
