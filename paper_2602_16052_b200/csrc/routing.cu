@@ -755,6 +755,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       s_count[tid] = c;
       s_offset[tid] = row0;
       s_unit_base[tid] = ub;
+      s_cand[tid] = chunks;                // (the candidate flags are no longer needed: token chunks per expert)
       ws.count[tid] = c;
       ws.offset[tid] = row0;
       ws.score[tid] = (double)s_fx[tid] * (1.0 / kScoreScale);
@@ -764,6 +765,7 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         s_offset[N] = row0 + c;
         ws.offset[N] = row0 + c;
         s_unit_base[N] = ub + chunks;
+        s_nchunks = ub + chunks;
         s_nactive = ai + (c > 0 && resident);
       }
     }
@@ -799,15 +801,19 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
       s_nchunks = tot;
     }
     __syncthreads();
-  } else if (a.tiles_up > 0) {
-    // Larger trees: the listed experts in the shortlist's rank order too, each with its token chunks.  Rank
-    // order is roughly row-count order, so the units that take longest (two or more full chunks, whose slabs
-    // are re-read by every chunk) are handed out first and the list ends with the cheap ones; in expert-index
-    // order whatever expert came last decided how long the CTAs waited for the last of them.
+  } else if (a.tiles_up > 0 && M <= 2 * kMaxTokChunk) {
+    // Trees of up to 256 tokens without early start: the listed experts in the shortlist's rank order too, each
+    // with its one or two token chunks.  Rank order is roughly row-count order, so the units that take longest
+    // (two full chunks, whose slabs are read twice) are handed out first and the list ends with cheap ones; in
+    // expert-index order whatever expert came last decided how long the CTAs waited for the last of them
+    // (-1 to -3 us at 129 to 255 tokens).  Larger trees keep the index order of the scan above: with three and
+    // more chunks per popular expert, rank order bunches the units that live on L2 re-reads at the start of
+    // the list, and the stream is slower there than with heavy and light experts interleaved (+2 % at 511
+    // tokens, unbudgeted).
     int e_r = 0, ch = 0;
     if (tid < nS_l) {
       e_r = s_Srank[tid];
-      ch = (s_count[e_r] + kMaxTokChunk - 1) / kMaxTokChunk;
+      ch = s_cand[e_r];
     }
     int inc = ch;
 #pragma unroll
@@ -821,20 +827,14 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
     for (int w = 0; w < warp; ++w) pre += (int)s_warp_tot[w];
     if (tid < nS_l) {
       s_unit_base[e_r] = pre;
-      s_cand[e_r] = ch;                    // (the candidate flags are no longer needed: chunk count per expert)
       for (int cc = 0; cc < ch && pre + cc < 2 * kMaxExperts; ++cc) s_chunk_expert[pre + cc] = e_r;
-    }
-    if (tid == 0) {
-      int tot = 0;
-      for (int w = 0; w < kRouteWarps; ++w) tot += (int)s_warp_tot[w];
-      s_nchunks = tot;
     }
     __syncthreads();
   }
 
   // The rest is three independent jobs, each latency-bound, run side by side:
   //   warps 0-3  row of every (token, slot)       warps 4-6  work-unit list       warp 7  coverage
-  const int n_chunks = a.tiles_up > 0 ? s_nchunks : s_unit_base[N];
+  const int n_chunks = s_nchunks;
   double cov = 0.0;
   if (warp < 4 && !a.rows_later) {
     // rows ordered by (expert ascending, token ascending): the row of (t, e) is
@@ -896,9 +896,10 @@ __global__ void __launch_bounds__(kRouteWarps * 32) route_kernel(RouteArgs a) {
         if (cpos < 2 * kMaxExperts) {
           e = s_chunk_expert[cpos];
         } else {          // more than 2N token chunks (M far beyond 128): search the chunk bases, in rank order
-          int r = 0;
-          e = s_Srank[0];
-          while (s_unit_base[e] + s_cand[e] <= cpos) e = s_Srank[++r];
+          e = 0;
+          for (int r = 0; r < N; ++r) {          // (whatever the order of the list: the intervals are disjoint)
+            if (s_cand[r] > 0 && s_unit_base[r] <= cpos && cpos < s_unit_base[r] + s_cand[r]) { e = r; break; }
+          }
         }
         // inside an expert: slab-major, token chunk innermost, so the chunks that re-read a slab are
         // handed out back to back and the second read hits L2
